@@ -1,0 +1,225 @@
+/*
+ * ap_serving.h -- C ABI of the paged-KV serving-iteration library (sm_100a).
+ *
+ * One continuous-batching serving iteration over a ragged batch: the new
+ * tokens' K/V are appended into a paged KV pool through per-sequence block
+ * tables, then every new token attends its sequence's context with
+ * grouped-query attention.  Sequences with one new token are decode steps,
+ * sequences with more are prefill chunks (causal inside the chunk).
+ *
+ * Where the operations come from.  The paper treats this iteration as the unit
+ * of work whose batch composition the scheduling policy decides and models it
+ * only by cost: continuous batching and per-operator time (Sec. 5.3 "Serving
+ * simulator"); a decode step k attends a context of k tokens including the new
+ * one, prefill is the separate longer-query operation (App. B, Eq.
+ * "serve-latency"); attention heads A_z, KV heads K_z <= A_z, head dimension
+ * d_z (App. B, model description); the KV cache is a finite pool counted in
+ * tokens (App. B Eq. "oom", theta = 0.8; App. C.2 "token-capacity limits");
+ * KV caches are relocatable (Sec. 4.1, Phase 2), hence block-table
+ * indirection; paged KV memory and chunked prefill are the data-plane
+ * techniques of the served systems (App. H).  The arithmetic itself is the
+ * textbook definition:
+ *     x_j = scale * <q, k_j>, j = 0..p;  out = softmax(x) V;  lse = ln sum_j e^{x_j}.
+ *
+ * Conventions
+ *   - All functions return int: AP_OK (0) or a negative ap_status.  Nothing
+ *     aborts, throws or traps the GPU.  Host-side validation happens before
+ *     any launch.
+ *   - "host" / "device" on a pointer says which memory it must point to.
+ *   - bf16 tensors are passed as void* (16-bit storage); page size is 16.
+ *   - Layouts (row-major, innermost last):
+ *         pool planes  K, V : [num_pages][num_kv_heads][16][head_dim]  bf16
+ *         q, out            : [N_new][num_q_heads][head_dim]           bf16
+ *         k_new, v_new      : [N_new][num_kv_heads][head_dim]          bf16
+ *         lse               : [N_new][num_q_heads]                     fp32, natural log
+ *     N_new = sum of q_lens; rows of all sequences are concatenated in batch
+ *     order.  q head h uses kv head h / (num_q_heads / num_kv_heads).
+ *   - Calls taking a stream are asynchronous and stream-ordered: ap_kv_append
+ *     followed by ap_attention_iteration on the same stream needs no sync.
+ *   - A plan must outlive the launches that use it (destroy it after the stream
+ *     has passed them, or after ap_last_device_status).
+ */
+#ifndef AP_SERVING_H
+#define AP_SERVING_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum ap_status {
+    AP_OK = 0,
+    AP_ERR_INVALID_ARG = -1,
+    AP_ERR_OUT_OF_PAGES = -2,
+    AP_ERR_BAD_BLOCK_TABLE = -3,
+    AP_ERR_WORKSPACE_TOO_SMALL = -4,
+    AP_ERR_CUDA = -5,
+    AP_ERR_TIMEOUT = -6,
+    AP_ERR_UNSUPPORTED = -7
+};
+
+typedef struct ap_kv_pool ap_kv_pool; /* opaque */
+typedef struct ap_plan ap_plan;       /* opaque */
+
+/* ------------------------------------------------------------------ pool -- */
+
+/*
+ * KV page pool (finite token capacity: App. B Eq. "oom", App. C.2).
+ * k_base/v_base: device, each ap_kv_pool_bytes() long and 1024-byte aligned,
+ * owned by the caller; or both NULL, then the library allocates (and zero
+ * fills) and frees them.  head_dim is 64 or 128; page_size must be 16;
+ * num_q_heads / num_kv_heads may be 1..8 (given per batch).
+ */
+typedef struct ap_pool_desc {
+    int32_t num_pages;
+    int32_t page_size;
+    int32_t num_kv_heads;
+    int32_t head_dim;
+    void *k_base; /* device or NULL */
+    void *v_base; /* device or NULL */
+    int32_t device;
+} ap_pool_desc;
+
+/* Bytes of ONE plane (K or V) for this description; 0 if the description is invalid. */
+size_t ap_kv_pool_bytes(const ap_pool_desc *desc);
+
+/*
+ * Creates the pool handle on desc->device: free list with all pages free in
+ * ascending order, tensor maps over both planes, a device status word.
+ * desc->device < 0 (with both bases NULL) creates a HOST-ONLY pool: the page
+ * allocator, ap_plan_create and ap_plan_export work (planning for 148 SMs);
+ * every call that would launch returns AP_ERR_CUDA.
+ * Errors: INVALID_ARG (bad sizes, one base NULL, misaligned), UNSUPPORTED
+ * (head_dim/page_size), CUDA (no device, allocation failure). */
+int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc);
+
+/* Frees the handle and only what the library allocated.  Synchronises the device. */
+int ap_kv_pool_destroy(ap_kv_pool *pool);
+
+/* Device addresses of the planes (caller's or the library's). */
+void *ap_kv_pool_k_base(const ap_kv_pool *pool);
+void *ap_kv_pool_v_base(const ap_kv_pool *pool);
+
+/* Host page allocator (per-request page ownership; pages are relocatable units,
+ * Sec. 4.1 Phase 2).  alloc is all-or-nothing: OUT_OF_PAGES leaves the free
+ * list unchanged.  out_ids / ids: host.  free of a page that is not allocated,
+ * out of range or repeated in the call -> INVALID_ARG, nothing freed. */
+int ap_kv_pool_alloc_pages(ap_kv_pool *pool, int32_t n, int32_t *out_ids);
+int ap_kv_pool_free_pages(ap_kv_pool *pool, int32_t n, const int32_t *ids);
+/* Shuffles the order in which FREE pages will be handed out (Fisher-Yates on a
+ * splitmix64 stream).  Allocated pages are unaffected. */
+int ap_kv_pool_seed_free_list(ap_kv_pool *pool, uint64_t seed);
+int32_t ap_kv_pool_num_free(const ap_kv_pool *pool);
+
+/* ------------------------------------------------------------------ plan -- */
+
+/*
+ * One iteration's batch (Sec. 5.3: the batch the policy composed).
+ * All arrays are HOST memory and are only read during ap_plan_create.
+ */
+typedef struct ap_batch_desc {
+    int32_t batch;               /* number of sequences B (>= 0) */
+    int32_t num_q_heads;         /* multiple of the pool's num_kv_heads, ratio 1..8 */
+    const int32_t *q_lens;       /* [B] new tokens this iteration: 0 skipped, 1 decode, >1 prefill chunk */
+    const int32_t *ctx_lens;     /* [B] context length INCLUDING this iteration's new tokens */
+    const int32_t *block_tables; /* [B][table_stride] logical -> physical page; entries past ceil(ctx/16) are never read */
+    int32_t table_stride;
+    float softmax_scale;         /* <= 0 selects 1/sqrt(head_dim) */
+} ap_batch_desc;
+
+/*
+ * Validates the batch and builds the device work lists (append destinations,
+ * split-K decode items balanced over the SMs, LSE-merge entries, prefill
+ * tiles), uploaded with one asynchronous copy on `stream`.
+ * Validation: 0 <= q_len <= ctx_len; table_stride >= ceil(ctx_len/16) for every
+ * sequence with q_len > 0; every used entry in [0, num_pages)
+ * (BAD_BLOCK_TABLE); no two appended token slots alias (BAD_BLOCK_TABLE);
+ * head ratio 1..8 (UNSUPPORTED).  Pages shared between sequences for reading
+ * are legal.  On error *out is NULL and nothing was launched.
+ */
+int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *batch, void *stream);
+int ap_plan_destroy(ap_plan *plan);
+
+/* Bytes of caller-provided device workspace (split-K partials) that
+ * ap_attention_iteration needs for this plan; may be 0. */
+size_t ap_plan_workspace_bytes(const ap_plan *plan);
+
+typedef struct ap_plan_info {
+    int64_t n_new;           /* rows of q / k_new / v_new / out */
+    int64_t kv_tokens;       /* sum of ctx_len over sequences with q_len > 0 */
+    int64_t decode_rows;     /* sequences with q_len == 1 */
+    int64_t prefill_seqs;    /* sequences with q_len > 1 */
+    int64_t prefill_pairs;   /* unmasked (query row, key) pairs of the prefill chunks, one head */
+    int64_t decode_items;    /* split-K work items */
+    int64_t decode_ctas;     /* persistent CTAs of the decode kernel */
+    int64_t merge_entries;   /* (row, kv head) results assembled from > 1 partial */
+    int64_t prefill_tiles;   /* work units of the prefill kernel */
+    int64_t launches_append; /* kernels ap_kv_append launches for this plan */
+    int64_t launches_attention; /* kernels ap_attention_iteration launches for this plan */
+} ap_plan_info;
+int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
+
+/*
+ * Host copy of the work lists a plan uploads, for inspection and tests.  The
+ * blob is an int32 array; the layout gives the offset (in int32 units) of each
+ * section:
+ *   append_dst    [n_new]             page*16 + slot of every new token row
+ *   bt_flat       [n_bt]              used block-table entries, sequences with q_len > 0 concatenated
+ *   decode_items  [decode_items][8]   q_row, kv_head, bt_offset, page_begin, page_count, kv_len, part_slot, 0
+ *   cta_begin     [n_cta_begin]       item range of decode CTA c is [cta_begin[c], cta_begin[c+1])
+ *   merge_entries [merge_entries][4]  q_row, kv_head, part_begin, part_count
+ *   prefill_tiles [prefill_tiles][8]  q_row0, rows, q_head, kv_head, bt_offset, pos0, ctx_len, 0
+ * blob: host, capacity_ints >= layout.total_ints, or NULL to query the layout only.
+ */
+typedef struct ap_plan_layout {
+    int64_t total_ints, append_dst, bt_flat, decode_items, cta_begin, merge_entries, prefill_tiles;
+    int64_t n_bt, n_cta_begin;
+} ap_plan_layout;
+int ap_plan_export(const ap_plan *plan, int32_t *blob, size_t capacity_ints, ap_plan_layout *layout);
+
+/* --------------------------------------------------------------- kernels -- */
+
+/*
+ * KV append (App. B Eq. "serve-latency": every step extends the context).
+ * Token t of sequence s sits at position p = ctx_len - q_len + t and is copied,
+ * bit for bit, to K/V[block_table[s][p/16]][kv_head][p%16][:].
+ * k_new, v_new: device, [N_new][num_kv_heads][head_dim] bf16, 16-byte aligned.
+ */
+int ap_kv_append(ap_kv_pool *pool, const ap_plan *plan, const void *k_new, const void *v_new,
+                 void *stream);
+
+/*
+ * Attention for every new token of the batch (decode rows: split-K
+ * flash-decoding + LSE merge; prefill chunks: causal tiled attention on
+ * tcgen05 tensor cores).  The pool must already hold the iteration's tokens.
+ * q, out: device, 16-byte aligned; lse: device or NULL; workspace: device,
+ * 256-byte aligned, at least ap_plan_workspace_bytes() (else
+ * WORKSPACE_TOO_SMALL), contents undefined before and after.
+ */
+int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
+                           float *lse, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The whole iteration from HOST buffers: plan, host->device copies of q,
+ * k_new, v_new, append, attention, device->host copy of out (and lse if not
+ * NULL), and a stream synchronisation.  Staging buffers belong to the pool and
+ * grow on demand.  q_host ... lse_host: host (pinned memory makes the copies
+ * asynchronous).  Returns the device status after the sync.
+ */
+int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, const void *q_host,
+                              const void *k_new_host, const void *v_new_host, void *out_host,
+                              float *lse_host, void *stream);
+
+/* Synchronises `stream` and returns (and clears) the device status word:
+ * AP_OK, AP_ERR_BAD_BLOCK_TABLE (a kernel met an out-of-range page id) or
+ * AP_ERR_TIMEOUT (a bounded wait inside a kernel ran out). */
+int ap_last_device_status(ap_kv_pool *pool, void *stream);
+
+const char *ap_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AP_SERVING_H */

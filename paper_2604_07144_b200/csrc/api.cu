@@ -1,0 +1,610 @@
+// Host side of the serving-iteration library: pool, page allocator, planner,
+// dispatch.  Every entry point validates on the host and returns a status;
+// nothing here (or in the kernels) aborts or traps.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace ap;
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; (void)cudaGetLastError(); }
+        ok = cudaSetDevice(dev) == cudaSuccess;
+        if (!ok) (void)cudaGetLastError();
+    }
+    ~DeviceGuard() {
+        if (prev >= 0 && ok) (void)cudaSetDevice(prev);
+    }
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool desc_valid(const ap_pool_desc *d) {
+    return d && d->num_pages > 0 && d->num_kv_heads > 0 && d->head_dim > 0 && d->page_size > 0;
+}
+
+// splitmix64: public-domain mixing function used as a counter-based stream.
+inline uint64_t splitmix64(uint64_t &state) {
+    uint64_t z = (state += 0x9E3779B97F4A7C15ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+void release_plan_buffer(PlanBuffer &b) {
+    if (b.uploaded) (void)cudaEventDestroy(b.uploaded);
+    if (b.host) (void)cudaFreeHost(b.host);
+    if (b.dev) (void)cudaFree(b.dev);
+    b = PlanBuffer{};
+}
+
+int acquire_plan_buffer(ap_kv_pool *pool, size_t n_ints, PlanBuffer *out) {
+    for (size_t i = 0; i < pool->plan_buffers.size(); ++i) {
+        if (pool->plan_buffers[i].capacity >= n_ints) {
+            *out = pool->plan_buffers[i];
+            pool->plan_buffers.erase(pool->plan_buffers.begin() + (long)i);
+            // the previous upload from this staging area must have been consumed
+            if (cudaEventSynchronize(out->uploaded) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return AP_ERR_CUDA;
+            }
+            return AP_OK;
+        }
+    }
+    PlanBuffer b;
+    b.capacity = std::max<size_t>(n_ints + n_ints / 2, 4096);
+    if (cudaMallocHost((void **)&b.host, b.capacity * sizeof(int32_t)) != cudaSuccess ||
+        cudaMalloc((void **)&b.dev, b.capacity * sizeof(int32_t)) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b.uploaded, cudaEventDisableTiming) != cudaSuccess) {
+        (void)cudaGetLastError();
+        release_plan_buffer(b);
+        return AP_ERR_CUDA;
+    }
+    *out = b;
+    return AP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ap_status_string(int status) {
+    switch (status) {
+        case AP_OK: return "ok";
+        case AP_ERR_INVALID_ARG: return "invalid argument";
+        case AP_ERR_OUT_OF_PAGES: return "out of KV pages";
+        case AP_ERR_BAD_BLOCK_TABLE: return "bad block table";
+        case AP_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case AP_ERR_CUDA: return "CUDA error";
+        case AP_ERR_TIMEOUT: return "device wait timed out";
+        case AP_ERR_UNSUPPORTED: return "unsupported configuration";
+        default: return "unknown status";
+    }
+}
+
+size_t ap_kv_pool_bytes(const ap_pool_desc *d) {
+    if (!desc_valid(d)) return 0;
+    return (size_t)d->num_pages * (size_t)d->num_kv_heads * (size_t)d->page_size *
+           (size_t)d->head_dim * 2u;
+}
+
+int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
+    if (!out) return AP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!desc_valid(desc)) return AP_ERR_INVALID_ARG;
+    if (desc->page_size != kPageSize) return AP_ERR_UNSUPPORTED;
+    if (desc->head_dim != 64 && desc->head_dim != 128) return AP_ERR_UNSUPPORTED;
+    if ((desc->k_base == nullptr) != (desc->v_base == nullptr)) return AP_ERR_INVALID_ARG;
+    if (((uintptr_t)desc->k_base | (uintptr_t)desc->v_base) & 1023u) return AP_ERR_INVALID_ARG;
+    // the tensor maps address 8-row groups with a 32-bit extent
+    if ((int64_t)desc->num_pages * desc->num_kv_heads * 2 >= (int64_t)1 << 31) return AP_ERR_UNSUPPORTED;
+
+    if (desc->device < 0) {
+        // host-only pool: allocator and planner work, nothing can be launched
+        if (desc->k_base) return AP_ERR_INVALID_ARG;
+        ap_kv_pool *hp = new (std::nothrow) ap_kv_pool();
+        if (!hp) return AP_ERR_CUDA;
+        hp->desc = *desc;
+        hp->sm_count = 148;
+        hp->free_list.resize((size_t)desc->num_pages);
+        for (int32_t i = 0; i < desc->num_pages; ++i) hp->free_list[(size_t)i] = desc->num_pages - 1 - i;
+        hp->allocated.assign((size_t)desc->num_pages, 0);
+        *out = hp;
+        return AP_OK;
+    }
+
+    DeviceGuard guard(desc->device);
+    if (!guard.ok) return AP_ERR_CUDA;
+
+    ap_kv_pool *p = new (std::nothrow) ap_kv_pool();
+    if (!p) return AP_ERR_CUDA;
+    p->desc = *desc;
+    int rc = AP_OK;
+    do {
+        if (cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess) {
+            rc = AP_ERR_CUDA;
+            break;
+        }
+        const size_t bytes = ap_kv_pool_bytes(desc);
+        if (!desc->k_base) {
+            p->owns_planes = true;
+            if (cudaMalloc(&p->desc.k_base, bytes) != cudaSuccess ||
+                cudaMalloc(&p->desc.v_base, bytes) != cudaSuccess ||
+                cudaMemset(p->desc.k_base, 0, bytes) != cudaSuccess ||
+                cudaMemset(p->desc.v_base, 0, bytes) != cudaSuccess) {
+                rc = AP_ERR_CUDA;
+                break;
+            }
+        }
+        if (cudaMalloc((void **)&p->d_status, sizeof(int)) != cudaSuccess ||
+            cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) {
+            rc = AP_ERR_CUDA;
+            break;
+        }
+        rc = encode_pool_tensor_map(&p->k_map, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
+        if (rc != AP_OK) break;
+        rc = encode_pool_tensor_map(&p->v_map, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
+        if (rc != AP_OK) break;
+        p->free_list.resize((size_t)desc->num_pages);
+        for (int32_t i = 0; i < desc->num_pages; ++i) p->free_list[(size_t)i] = desc->num_pages - 1 - i;
+        p->allocated.assign((size_t)desc->num_pages, 0);
+    } while (false);
+    if (rc != AP_OK) {
+        (void)cudaGetLastError();
+        ap_kv_pool_destroy(p);
+        return rc;
+    }
+    *out = p;
+    return AP_OK;
+}
+
+int ap_kv_pool_destroy(ap_kv_pool *pool) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) { delete pool; return AP_OK; }
+    DeviceGuard guard(pool->desc.device);
+    if (guard.ok) (void)cudaDeviceSynchronize();
+    for (auto &b : pool->plan_buffers) release_plan_buffer(b);
+    if (pool->stage_dev) (void)cudaFree(pool->stage_dev);
+    if (pool->d_status) (void)cudaFree(pool->d_status);
+    if (pool->owns_planes) {
+        if (pool->desc.k_base) (void)cudaFree(pool->desc.k_base);
+        if (pool->desc.v_base) (void)cudaFree(pool->desc.v_base);
+    }
+    (void)cudaGetLastError();
+    delete pool;
+    return AP_OK;
+}
+
+void *ap_kv_pool_k_base(const ap_kv_pool *pool) { return pool ? pool->desc.k_base : nullptr; }
+void *ap_kv_pool_v_base(const ap_kv_pool *pool) { return pool ? pool->desc.v_base : nullptr; }
+
+int ap_kv_pool_alloc_pages(ap_kv_pool *pool, int32_t n, int32_t *out_ids) {
+    if (!pool || n < 0 || (n > 0 && !out_ids)) return AP_ERR_INVALID_ARG;
+    if ((size_t)n > pool->free_list.size()) return AP_ERR_OUT_OF_PAGES;
+    for (int32_t i = 0; i < n; ++i) {
+        int32_t id = pool->free_list.back();
+        pool->free_list.pop_back();
+        pool->allocated[(size_t)id] = 1;
+        out_ids[i] = id;
+    }
+    return AP_OK;
+}
+
+int ap_kv_pool_free_pages(ap_kv_pool *pool, int32_t n, const int32_t *ids) {
+    if (!pool || n < 0 || (n > 0 && !ids)) return AP_ERR_INVALID_ARG;
+    // first pass validates (and detects repeats inside the call), second frees
+    for (int32_t i = 0; i < n; ++i) {
+        int32_t id = ids[i];
+        if (id < 0 || id >= pool->desc.num_pages || pool->allocated[(size_t)id] != 1) {
+            for (int32_t j = 0; j < i; ++j) pool->allocated[(size_t)ids[j]] = 1;
+            return AP_ERR_INVALID_ARG;
+        }
+        pool->allocated[(size_t)id] = 2;  // marked within this call
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        pool->allocated[(size_t)ids[i]] = 0;
+        pool->free_list.push_back(ids[i]);
+    }
+    return AP_OK;
+}
+
+int ap_kv_pool_seed_free_list(ap_kv_pool *pool, uint64_t seed) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    auto &f = pool->free_list;
+    uint64_t state = seed;
+    for (size_t i = f.size(); i > 1; --i) {
+        size_t j = (size_t)(splitmix64(state) % (uint64_t)i);
+        std::swap(f[i - 1], f[j]);
+    }
+    return AP_OK;
+}
+
+int32_t ap_kv_pool_num_free(const ap_kv_pool *pool) {
+    return pool ? (int32_t)pool->free_list.size() : 0;
+}
+
+// ---------------------------------------------------------------- planner --
+
+int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void *stream) {
+    if (!out) return AP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!pool || !b || b->batch < 0 || b->num_q_heads <= 0) return AP_ERR_INVALID_ARG;
+    if (b->batch > 0 && (!b->q_lens || !b->ctx_lens || !b->block_tables || b->table_stride <= 0))
+        return AP_ERR_INVALID_ARG;
+    const int Hkv = pool->desc.num_kv_heads, d = pool->desc.head_dim;
+    if (b->num_q_heads % Hkv != 0) return AP_ERR_INVALID_ARG;
+    const int G = b->num_q_heads / Hkv;
+    if (G < 1 || G > 8) return AP_ERR_UNSUPPORTED;
+    const int B = b->batch;
+    const int32_t num_pages = pool->desc.num_pages;
+
+    // ---- validation + row bookkeeping
+    int64_t n_new = 0, kv_tokens = 0, bt_total = 0, pairs = 0;
+    int64_t decode_rows = 0, prefill_seqs = 0;
+    for (int s = 0; s < B; ++s) {
+        const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
+        if (ql < 0 || cl < 0 || ql > cl) return AP_ERR_INVALID_ARG;
+        if (ql == 0) continue;
+        const int64_t need = ((int64_t)cl + kPageSize - 1) / kPageSize;
+        if (need > b->table_stride) return AP_ERR_INVALID_ARG;
+        const int32_t *row = b->block_tables + (size_t)s * (size_t)b->table_stride;
+        for (int64_t i = 0; i < need; ++i)
+            if (row[i] < 0 || row[i] >= num_pages) return AP_ERR_BAD_BLOCK_TABLE;
+        n_new += ql;
+        kv_tokens += cl;
+        bt_total += need;
+        if (ql == 1) ++decode_rows; else ++prefill_seqs;
+        if (ql > 1) pairs += (int64_t)ql * (cl - ql) + (int64_t)ql * (ql + 1) / 2;
+    }
+    if (n_new > (int64_t)1 << 30) return AP_ERR_UNSUPPORTED;
+
+    std::vector<int32_t> append_dst((size_t)n_new);
+    std::vector<int32_t> bt_off((size_t)B, 0);
+    std::vector<int32_t> row0((size_t)B + 1, 0);
+    {
+        int64_t r = 0, off = 0;
+        for (int s = 0; s < B; ++s) {
+            row0[(size_t)s] = (int32_t)r;
+            const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
+            if (ql == 0) continue;
+            bt_off[(size_t)s] = (int32_t)off;
+            off += ((int64_t)cl + kPageSize - 1) / kPageSize;
+            const int32_t *row = b->block_tables + (size_t)s * (size_t)b->table_stride;
+            for (int32_t t = 0; t < ql; ++t) {
+                const int32_t p = cl - ql + t;
+                append_dst[(size_t)r++] = row[p / kPageSize] * kPageSize + p % kPageSize;
+            }
+        }
+        row0[(size_t)B] = (int32_t)r;
+        // no two appended slots may alias
+        std::vector<int32_t> sorted(append_dst);
+        std::sort(sorted.begin(), sorted.end());
+        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AP_ERR_BAD_BLOCK_TABLE;
+    }
+
+    // ---- decode: cut the (row, kv head) page streams into per-CTA item lists
+    const int max_ctas = std::max(1, pool->sm_count * decode_ctas_per_sm(d));
+    constexpr int kItemCost = 2;          // fixed per-item cost, in page units
+    constexpr int kStage = kDecodePagesPerStage;
+    std::vector<DecodeItem> items;
+    std::vector<int32_t> cta_begin;
+    std::vector<MergeEntry> merges;
+    int n_slots = 0;
+    if (decode_rows > 0) {
+        int64_t total_cost = 0;
+        for (int s = 0; s < B; ++s)
+            if (b->q_lens[s] == 1)
+                total_cost += (int64_t)Hkv * (((int64_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize + kItemCost);
+        int64_t target = std::max<int64_t>((total_cost + max_ctas - 1) / max_ctas, 2 * kStage + kItemCost);
+        for (int attempt = 0; attempt < 64; ++attempt) {
+            items.clear(); cta_begin.clear(); merges.clear(); n_slots = 0;
+            cta_begin.push_back(0);
+            int64_t cap = target;
+            auto next_cta = [&]() {
+                if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
+                cap = target;
+            };
+            for (int s = 0; s < B; ++s) {
+                if (b->q_lens[s] != 1) continue;
+                const int32_t cl = b->ctx_lens[s];
+                const int32_t pages = (cl + kPageSize - 1) / kPageSize;
+                for (int g = 0; g < Hkv; ++g) {
+                    int32_t rem = pages, pb = 0;
+                    const size_t first = items.size();
+                    while (rem > 0) {
+                        int64_t avail = cap - kItemCost;
+                        if (avail < kStage && avail < rem) { next_cta(); continue; }
+                        int32_t take = (int32_t)std::min<int64_t>(rem, avail);
+                        if (take < rem) take = take / kStage * kStage;
+                        DecodeItem it{};
+                        it.q_row = row0[(size_t)s];
+                        it.kv_head = g;
+                        it.bt_offset = bt_off[(size_t)s];
+                        it.page_begin = pb;
+                        it.page_count = take;
+                        it.kv_len = cl;
+                        it.part_slot = -1;
+                        items.push_back(it);
+                        cap -= take + kItemCost;
+                        pb += take;
+                        rem -= take;
+                        if (cap < kItemCost + kStage) next_cta();
+                    }
+                    if (items.size() - first > 1) {
+                        MergeEntry m{row0[(size_t)s], g, n_slots, (int32_t)(items.size() - first)};
+                        merges.push_back(m);
+                        for (size_t i = first; i < items.size(); ++i) items[i].part_slot = n_slots++;
+                    }
+                }
+            }
+            if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
+            if ((int)cta_begin.size() - 1 <= max_ctas) break;
+            target += std::max<int64_t>(1, target / 256);
+        }
+    }
+    const int n_ctas = cta_begin.empty() ? 0 : (int)cta_begin.size() - 1;
+
+    // ---- prefill tiles, longest first
+    std::vector<PrefillTile> tiles;
+    for (int s = 0; s < B; ++s) {
+        const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
+        if (ql <= 1) continue;
+        for (int32_t t0 = 0; t0 < ql; t0 += 128) {
+            for (int h = 0; h < b->num_q_heads; ++h) {
+                PrefillTile t{};
+                t.q_row0 = row0[(size_t)s] + t0;
+                t.rows = std::min(128, ql - t0);
+                t.q_head = h;
+                t.kv_head = h / G;
+                t.bt_offset = bt_off[(size_t)s];
+                t.pos0 = cl - ql + t0;
+                t.ctx_len = cl;
+                tiles.push_back(t);
+            }
+        }
+    }
+    std::stable_sort(tiles.begin(), tiles.end(), [](const PrefillTile &a, const PrefillTile &c) {
+        return a.pos0 + a.rows > c.pos0 + c.rows;
+    });
+
+    // ---- blob layout (int32 units, every section 32-byte aligned)
+    auto sec = [](size_t &cursor, size_t n_ints) {
+        size_t at = cursor;
+        cursor = (cursor + n_ints + 7) / 8 * 8;
+        return at;
+    };
+    size_t cursor = 0;
+    const size_t o_append = sec(cursor, (size_t)n_new);
+    const size_t o_bt = sec(cursor, (size_t)bt_total);
+    const size_t o_items = sec(cursor, items.size() * 8);
+    const size_t o_cta = sec(cursor, cta_begin.size());
+    const size_t o_merge = sec(cursor, merges.size() * 4);
+    const size_t o_tiles = sec(cursor, tiles.size() * 8);
+    const size_t total_ints = std::max<size_t>(cursor, 8);
+
+    ap_plan *plan = new (std::nothrow) ap_plan();
+    if (!plan) return AP_ERR_CUDA;
+    plan->blob.assign(total_ints, 0);
+    int32_t *h = plan->blob.data();
+    if (n_new) std::memcpy(h + o_append, append_dst.data(), (size_t)n_new * 4);
+    for (int s = 0; s < B; ++s) {
+        if (b->q_lens[s] == 0) continue;
+        const size_t need = ((size_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize;
+        std::memcpy(h + o_bt + bt_off[(size_t)s], b->block_tables + (size_t)s * (size_t)b->table_stride, need * 4);
+    }
+    if (!items.empty()) std::memcpy(h + o_items, items.data(), items.size() * sizeof(DecodeItem));
+    if (!cta_begin.empty()) std::memcpy(h + o_cta, cta_begin.data(), cta_begin.size() * 4);
+    if (!merges.empty()) std::memcpy(h + o_merge, merges.data(), merges.size() * sizeof(MergeEntry));
+    if (!tiles.empty()) std::memcpy(h + o_tiles, tiles.data(), tiles.size() * sizeof(PrefillTile));
+    plan->layout.total_ints = (int64_t)total_ints;
+    plan->layout.append_dst = (int64_t)o_append;
+    plan->layout.bt_flat = (int64_t)o_bt;
+    plan->layout.decode_items = (int64_t)o_items;
+    plan->layout.cta_begin = (int64_t)o_cta;
+    plan->layout.merge_entries = (int64_t)o_merge;
+    plan->layout.prefill_tiles = (int64_t)o_tiles;
+    plan->layout.n_bt = bt_total;
+    plan->layout.n_cta_begin = (int64_t)cta_begin.size();
+
+    if (pool->desc.device >= 0) {
+        DeviceGuard guard(pool->desc.device);
+        if (!guard.ok) { delete plan; return AP_ERR_CUDA; }
+        int rc = acquire_plan_buffer(pool, total_ints, &plan->buf);
+        if (rc != AP_OK) { delete plan; return rc; }
+        std::memcpy(plan->buf.host, h, total_ints * 4);
+        cudaStream_t st = (cudaStream_t)stream;
+        if (cudaMemcpyAsync(plan->buf.dev, plan->buf.host, total_ints * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaEventRecord(plan->buf.uploaded, st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            pool->plan_buffers.push_back(plan->buf);
+            delete plan;
+            return AP_ERR_CUDA;
+        }
+    }
+
+    plan->pool = pool;
+    plan->num_q_heads = b->num_q_heads;
+    plan->group = G;
+    plan->scale = b->softmax_scale > 0.f ? b->softmax_scale : 1.0f / std::sqrt((float)d);
+    plan->n_part_slots = n_slots;
+    plan->d_append_dst = plan->buf.dev + o_append;
+    plan->d_bt_flat = plan->buf.dev + o_bt;
+    plan->d_items = (const DecodeItem *)(plan->buf.dev + o_items);
+    plan->d_cta_begin = plan->buf.dev + o_cta;
+    plan->d_merge = (const MergeEntry *)(plan->buf.dev + o_merge);
+    plan->d_tiles = (const PrefillTile *)(plan->buf.dev + o_tiles);
+    plan->ws.o_part_off = 0;
+    plan->ws.lse_part_off = align_up((size_t)n_slots * G * d * sizeof(float), 256);
+    plan->ws.bytes = n_slots ? plan->ws.lse_part_off + align_up((size_t)n_slots * G * sizeof(float), 256) : 0;
+
+    ap_plan_info &info = plan->info;
+    info.n_new = n_new;
+    info.kv_tokens = kv_tokens;
+    info.decode_rows = decode_rows;
+    info.prefill_seqs = prefill_seqs;
+    info.prefill_pairs = pairs;
+    info.decode_items = (int64_t)items.size();
+    info.decode_ctas = n_ctas;
+    info.merge_entries = (int64_t)merges.size();
+    info.prefill_tiles = (int64_t)tiles.size();
+    info.launches_append = n_new > 0 ? 1 : 0;
+    info.launches_attention = (items.empty() ? 0 : 1) + (merges.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
+    *out = plan;
+    return AP_OK;
+}
+
+int ap_plan_destroy(ap_plan *plan) {
+    if (!plan) return AP_ERR_INVALID_ARG;
+    if (plan->pool && plan->buf.dev) plan->pool->plan_buffers.push_back(plan->buf);
+    delete plan;
+    return AP_OK;
+}
+
+size_t ap_plan_workspace_bytes(const ap_plan *plan) { return plan ? plan->ws.bytes : 0; }
+
+int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info) {
+    if (!plan || !info) return AP_ERR_INVALID_ARG;
+    *info = plan->info;
+    return AP_OK;
+}
+
+int ap_plan_export(const ap_plan *plan, int32_t *blob, size_t capacity_ints, ap_plan_layout *layout) {
+    if (!plan || !layout) return AP_ERR_INVALID_ARG;
+    *layout = plan->layout;
+    if (blob) {
+        if (capacity_ints < plan->blob.size()) return AP_ERR_INVALID_ARG;
+        std::memcpy(blob, plan->blob.data(), plan->blob.size() * 4);
+    }
+    return AP_OK;
+}
+
+// --------------------------------------------------------------- dispatch --
+
+int ap_kv_append(ap_kv_pool *pool, const ap_plan *plan, const void *k_new, const void *v_new, void *stream) {
+    if (!pool || !plan || plan->pool != pool) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    if (plan->info.n_new == 0) return AP_OK;
+    if (!k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15u)) return AP_ERR_INVALID_ARG;
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    if (launch_kv_append(pool, plan, k_new, v_new, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return AP_ERR_CUDA;
+    }
+    return AP_OK;
+}
+
+int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
+                           void *workspace, size_t workspace_bytes, void *stream) {
+    if (!pool || !plan || plan->pool != pool) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    if (plan->info.n_new == 0) return AP_OK;
+    if (!q || !out || (((uintptr_t)q | (uintptr_t)out) & 15u)) return AP_ERR_INVALID_ARG;
+    if (plan->ws.bytes > 0) {
+        if (!workspace || workspace_bytes < plan->ws.bytes) return AP_ERR_WORKSPACE_TOO_SMALL;
+        if ((uintptr_t)workspace & 255u) return AP_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    float *o_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.o_part_off) : nullptr;
+    float *lse_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.lse_part_off) : nullptr;
+    cudaError_t e = cudaSuccess;
+    if (plan->info.decode_items > 0) e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+    if (e == cudaSuccess && plan->info.merge_entries > 0)
+        e = launch_lse_merge(pool, plan, o_part, lse_part, out, lse, st);
+    if (e == cudaSuccess && plan->info.prefill_tiles > 0) e = launch_prefill(pool, plan, q, out, lse, st);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return e == cudaErrorNotSupported ? AP_ERR_UNSUPPORTED : AP_ERR_CUDA;
+    }
+    return AP_OK;
+}
+
+int ap_last_device_status(ap_kv_pool *pool, void *stream) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int status = 0;
+    if (cudaMemcpyAsync(&status, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return AP_ERR_CUDA;
+    }
+    if (status != 0) {
+        if (cudaMemsetAsync(pool->d_status, 0, sizeof(int), st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return AP_ERR_CUDA;
+        }
+    }
+    return status;
+}
+
+int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, const void *q_host,
+                              const void *k_new_host, const void *v_new_host, void *out_host,
+                              float *lse_host, void *stream) {
+    if (!pool || !batch) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    ap_plan *plan = nullptr;
+    int rc = ap_plan_create(&plan, pool, batch, stream);
+    if (rc != AP_OK) return rc;
+    const size_t n = (size_t)plan->info.n_new;
+    if (n == 0) { ap_plan_destroy(plan); return AP_OK; }
+    if (!q_host || !k_new_host || !v_new_host || !out_host) { ap_plan_destroy(plan); return AP_ERR_INVALID_ARG; }
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) { ap_plan_destroy(plan); return AP_ERR_CUDA; }
+    const size_t d = (size_t)pool->desc.head_dim, Hq = (size_t)batch->num_q_heads, Hkv = (size_t)pool->desc.num_kv_heads;
+    const size_t q_bytes = align_up(n * Hq * d * 2, 256), kv_bytes = align_up(n * Hkv * d * 2, 256);
+    const size_t lse_bytes = align_up(n * Hq * 4, 256), ws_bytes = align_up(plan->ws.bytes, 256);
+    const size_t total = 2 * q_bytes + 2 * kv_bytes + lse_bytes + ws_bytes;
+    if (total > pool->stage_bytes) {
+        if (pool->stage_dev) {
+            (void)cudaDeviceSynchronize();
+            (void)cudaFree(pool->stage_dev);
+            pool->stage_dev = nullptr;
+            pool->stage_bytes = 0;
+        }
+        const size_t want = total + total / 4;
+        if (cudaMalloc(&pool->stage_dev, want) != cudaSuccess) {
+            (void)cudaGetLastError();
+            ap_plan_destroy(plan);
+            return AP_ERR_CUDA;
+        }
+        pool->stage_bytes = want;
+    }
+    char *base = (char *)pool->stage_dev;
+    void *dq = base, *dout = base + q_bytes, *dk = base + 2 * q_bytes, *dv = base + 2 * q_bytes + kv_bytes;
+    float *dlse = (float *)(base + 2 * q_bytes + 2 * kv_bytes);
+    void *dws = base + 2 * q_bytes + 2 * kv_bytes + lse_bytes;
+    bool ok = cudaMemcpyAsync(dq, q_host, n * Hq * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(dk, k_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(dv, v_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (ok) {
+        rc = ap_kv_append(pool, plan, dk, dv, stream);
+        if (rc == AP_OK) rc = ap_attention_iteration(pool, plan, dq, dout, dlse, dws, ws_bytes, stream);
+        if (rc == AP_OK) {
+            ok = cudaMemcpyAsync(out_host, dout, n * Hq * d * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+            if (ok && lse_host)
+                ok = cudaMemcpyAsync(lse_host, dlse, n * Hq * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        }
+    }
+    if (!ok) { (void)cudaGetLastError(); rc = AP_ERR_CUDA; }
+    const int dev_status = ap_last_device_status(pool, stream);  // synchronises the stream
+    ap_plan_destroy(plan);
+    return rc != AP_OK ? rc : dev_status;
+}
+
+}  // extern "C"

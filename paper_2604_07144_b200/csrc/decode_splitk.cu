@@ -1,0 +1,345 @@
+// Decode attention: split-K flash-decoding over paged KV (HBM-bound).
+//
+// A persistent CTA walks its list of work items; an item is the G query heads
+// of one kv head of one decode row over a contiguous range of the sequence's
+// pages.  One producer warp streams (page, kv head) tiles of K and V -- 4 KB
+// each, contiguous in HBM -- into a multi-stage shared-memory ring with TMA
+// (128-byte swizzle, completion on mbarriers) and runs ahead across item
+// boundaries, so the pipeline never drains while consumers finish an item.
+// Four consumer warps each own one page of a stage:
+//     S^T = K_page Q^T      (mma.sync m16n8k16: M = 16 tokens, N = 8 heads)
+//     online softmax over tokens (fp32, warp shuffles across the token lanes)
+//     O^T += V_page^T P^T   (M = 16 columns of d per tile, N = 8 heads)
+// so every MMA row is a real token and no accumulator register is padding.
+// At the end of an item the four warps' (m, l, O) are combined through shared
+// memory and written either as the final bf16 output (item covers the whole
+// context) or as an fp32 partial (o normalised, lse) for the merge kernel.
+#include <cuda_bf16.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace ap {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kConsumerWarps = 4;
+constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kPPS = kDecodePagesPerStage;
+static_assert(kPPS == kConsumerWarps, "one page of a stage per consumer warp");
+
+template <int D>
+struct DecodeCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kTileBytes = kPageSize * D * 2;            // one (page, head) tile of one plane
+    static constexpr int kQBytes = 8 * D * 2;                       // up to 8 query heads
+    static constexpr int kStageBytes = 2 * kPPS * kTileBytes + kQBytes;
+    static constexpr int kStages = D == 128 ? 5 : 8;
+    static constexpr int kORow = D + 4;                             // padded fp32 row of the merge buffer
+    static constexpr int kMergeWarpFloats = 8 * kORow + 16;         // O[8][D+4], m[8], l[8]
+    static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4;
+    static constexpr int kBarrierBytes = 2 * kStages * 8 + 16;
+    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kMergeBytes + kBarrierBytes;
+    static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte swizzle alignment");
+};
+
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up after ~2 s (or when another warp has flagged abort).
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+// byte offset of the 16-byte chunk `chunk` (0 .. D/8-1) of token `tok` (0..15)
+// inside a swizzled (page, head) tile: [token/8][half][token%8][64 elements]
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int tok, int chunk) {
+    return (uint32_t)((tok >> 3) * (1024 * (D / 64)) + (chunk >> 3) * 1024 + (tok & 7) * 128 +
+                      (((chunk & 7) ^ (tok & 7)) << 4));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecodeThreads, 1)
+decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                     const __nv_bfloat16 *__restrict__ q, const DecodeItem *__restrict__ items,
+                     const int32_t *__restrict__ cta_begin, const int32_t *__restrict__ bt_flat,
+                     float *__restrict__ o_part, float *__restrict__ lse_part, __nv_bfloat16 *__restrict__ out,
+                     float *__restrict__ lse_out, int Hq, int Hkv, int G, int num_pages, float scale_log2,
+                     int *status) {
+    using Cfg = DecodeCfg<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *stages = smem;
+    float *merge = (float *)(smem + Cfg::kStages * Cfg::kStageBytes);
+    uint64_t *full = (uint64_t *)((uint8_t *)merge + Cfg::kMergeBytes);
+    uint64_t *empty = full + Cfg::kStages;
+    volatile int *abort_flag = (volatile int *)(empty + Cfg::kStages);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int item_begin = cta_begin[blockIdx.x], item_end = cta_begin[blockIdx.x + 1];
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cfg::kStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kConsumerWarps);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    int stage = 0;
+    uint32_t phase = 0;
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------------------------------ producer --
+        if (lane == 0) {
+            prefetch_tensormap(&k_map);
+            prefetch_tensormap(&v_map);
+        }
+        for (int it = item_begin; it < item_end; ++it) {
+            const DecodeItem item = items[it];
+            const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
+            const int npages = item.page_count;
+            int32_t cur = lane < npages ? __ldg(bt + lane) : 0;
+            for (int p0 = 0; p0 < npages; p0 += 32) {
+                const int32_t nxt = p0 + 32 + lane < npages ? __ldg(bt + p0 + 32 + lane) : 0;
+                const int ngroup = min(32, npages - p0);
+                for (int s0 = 0; s0 < ngroup; s0 += kPPS) {
+                    const int n = min(kPPS, ngroup - s0);
+                    if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag)) {
+                        atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                        *abort_flag = 1;
+                        return;
+                    }
+                    int32_t page = __shfl_sync(0xffffffffu, cur, s0 + (lane & (kPPS - 1)));
+                    const bool first = (p0 == 0 && s0 == 0);
+                    uint8_t *st = stages + stage * Cfg::kStageBytes;
+                    if (lane == 0)
+                        mbar_arrive_expect_tx(&full[stage], (uint32_t)(n * 2 * Cfg::kTileBytes +
+                                                                      (first ? G * D * 2 : 0)));
+                    __syncwarp();
+                    if (lane < n) {
+                        if (page < 0 || page >= num_pages) {
+                            atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                            page = 0;
+                        }
+                        const int group = (page * Hkv + item.kv_head) * 2;
+                        tma_load_4d(st + lane * Cfg::kTileBytes, &k_map, &full[stage], 0, 0, 0, group);
+                        tma_load_4d(st + (kPPS + lane) * Cfg::kTileBytes, &v_map, &full[stage], 0, 0, 0, group);
+                    } else if (lane == kPPS && first) {
+                        bulk_load(st + 2 * kPPS * Cfg::kTileBytes,
+                                  q + ((size_t)item.q_row * Hq + (size_t)item.kv_head * G) * D,
+                                  (uint32_t)(G * D * 2), &full[stage]);
+                    }
+                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+                }
+                cur = nxt;
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------- consumers --
+    const int g = lane >> 2, t = lane & 3;
+    const float kLn2 = 0.6931471805599453f;
+    float *my_merge = merge + warp * Cfg::kMergeWarpFloats;
+
+    for (int it = item_begin; it < item_end; ++it) {
+        const DecodeItem item = items[it];
+        const int npages = item.page_count;
+        const int valid = min(item.kv_len, (item.page_begin + npages) * kPageSize) - item.page_begin * kPageSize;
+
+        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+        float o[D / 16][4];
+#pragma unroll
+        for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        uint32_t qf[D / 16][2];
+
+        for (int p0 = 0; p0 < npages; p0 += kPPS) {
+            if (!wait_or_abort(&full[stage], phase, abort_flag)) {
+                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                *abort_flag = 1;
+                return;
+            }
+            uint8_t *st = stages + stage * Cfg::kStageBytes;
+            if (p0 == 0) {
+                // Q^T as the B operand: b0 = Q[head g][16ks + 2t, +1], b1 = Q[head g][16ks + 8 + 2t, +1]
+                const uint32_t *qs = (const uint32_t *)(st + 2 * kPPS * Cfg::kTileBytes);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    qf[ks][0] = g < G ? qs[(g * D + ks * 16 + 2 * t) >> 1] : 0u;
+                    qf[ks][1] = g < G ? qs[(g * D + ks * 16 + 8 + 2 * t) >> 1] : 0u;
+                }
+            }
+            const int my_page = p0 + warp;
+            if (my_page < npages) {
+                const int tv = min(kPageSize, valid - my_page * kPageSize);   // valid tokens in this page (>= 1)
+                const uint32_t k_tile = smem_u32(st + warp * Cfg::kTileBytes);
+                uint8_t *v_ptr = st + (kPPS + warp) * Cfg::kTileBytes;
+                const uint32_t v_tile = smem_u32(v_ptr);
+                if (tv < kPageSize) {
+                    // slots past the context hold no token: clear their V rows so 0 * garbage cannot poison O
+                    for (int idx = lane; idx < (kPageSize - tv) * (D / 8); idx += 32) {
+                        const int tok = tv + idx / (D / 8), ch = idx % (D / 8);
+                        *(uint4 *)(v_ptr + tile_off<D>(tok, ch)) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
+                // ---- S^T = K Q^T : tokens (g, g+8) x heads (2t, 2t+1)
+                float s[4] = {0.f, 0.f, 0.f, 0.f};
+                {
+                    const int mat = lane >> 3, r = lane & 7;
+                    const int tok = (mat & 1) * 8 + r;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        uint32_t a[4];
+                        ldmatrix_x4(a, k_tile + tile_off<D>(tok, 2 * ks + (mat >> 1)));
+                        mma_bf16_16816(s, a[0], a[1], a[2], a[3], qf[ks][0], qf[ks][1]);
+                    }
+                }
+                if (g >= tv) s[0] = s[1] = -INFINITY;
+                if (g + 8 >= tv) s[2] = s[3] = -INFINITY;
+                float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+#pragma unroll
+                for (int sh = 4; sh <= 16; sh <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+                }
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                const float al0 = exp2_approx((m0 - mn0) * scale_log2), al1 = exp2_approx((m1 - mn1) * scale_log2);
+                const float ms0 = mn0 * scale_log2, ms1 = mn1 * scale_log2;
+                const float p0_ = exp2_approx(s[0] * scale_log2 - ms0), p1_ = exp2_approx(s[1] * scale_log2 - ms1);
+                const float p2_ = exp2_approx(s[2] * scale_log2 - ms0), p3_ = exp2_approx(s[3] * scale_log2 - ms1);
+                l0 = l0 * al0 + p0_ + p2_;
+                l1 = l1 * al1 + p1_ + p3_;
+                m0 = mn0;
+                m1 = mn1;
+#pragma unroll
+                for (int i = 0; i < D / 16; ++i) {
+                    o[i][0] *= al0; o[i][1] *= al1; o[i][2] *= al0; o[i][3] *= al1;
+                }
+                // P^T as the B operand: transpose the two 8x8 (token x head) blocks across the warp
+                const uint32_t b0 = movmatrix_trans(pack_bf16x2(p0_, p1_));
+                const uint32_t b1 = movmatrix_trans(pack_bf16x2(p2_, p3_));
+                // ---- O^T += V^T P^T : columns of d (16mt + g, + 8) x heads (2t, 2t+1)
+                {
+                    const int mat = lane >> 3, r = lane & 7;
+                    const int tok = (mat >> 1) * 8 + r;
+#pragma unroll
+                    for (int mt = 0; mt < D / 16; ++mt) {
+                        uint32_t a[4];
+                        ldmatrix_x4_trans(a, v_tile + tile_off<D>(tok, 2 * mt + (mat & 1)));
+                        mma_bf16_16816(o[mt], a[0], a[1], a[2], a[3], b0, b1);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty[stage]);
+            if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+        }
+
+        // ---- combine the four warps' (m, l, O)
+#pragma unroll
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+            l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
+        }
+#pragma unroll
+        for (int mt = 0; mt < D / 16; ++mt) {
+            my_merge[(2 * t) * Cfg::kORow + mt * 16 + g] = o[mt][0];
+            my_merge[(2 * t + 1) * Cfg::kORow + mt * 16 + g] = o[mt][1];
+            my_merge[(2 * t) * Cfg::kORow + mt * 16 + g + 8] = o[mt][2];
+            my_merge[(2 * t + 1) * Cfg::kORow + mt * 16 + g + 8] = o[mt][3];
+        }
+        if (g == 0) {
+            my_merge[8 * Cfg::kORow + 2 * t] = m0;
+            my_merge[8 * Cfg::kORow + 2 * t + 1] = m1;
+            my_merge[8 * Cfg::kORow + 8 + 2 * t] = l0;
+            my_merge[8 * Cfg::kORow + 8 + 2 * t + 1] = l1;
+        }
+        named_barrier_sync(1, kConsumerWarps * 32);
+        for (int idx = threadIdx.x; idx < G * D; idx += kConsumerWarps * 32) {
+            const int head = idx / D, col = idx % D;
+            float mstar = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w)
+                mstar = fmaxf(mstar, merge[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + head]);
+            float L = 0.f, acc = 0.f;
+#pragma unroll
+            for (int w = 0; w < kConsumerWarps; ++w) {
+                const float *mw = merge + w * Cfg::kMergeWarpFloats;
+                const float wt = exp2_approx((mw[8 * Cfg::kORow + head] - mstar) * scale_log2);
+                L += wt * mw[8 * Cfg::kORow + 8 + head];
+                acc += wt * mw[head * Cfg::kORow + col];
+            }
+            const float val = acc / L;
+            const float lse = (mstar * scale_log2 + log2f(L)) * kLn2;
+            if (item.part_slot < 0) {
+                const size_t row = (size_t)item.q_row * Hq + (size_t)item.kv_head * G + head;
+                out[row * D + col] = __float2bfloat16_rn(val);
+                if (col == 0 && lse_out) lse_out[row] = lse;
+            } else {
+                const size_t row = (size_t)item.part_slot * G + head;
+                o_part[row * D + col] = val;
+                if (col == 0) lse_part[row] = lse;
+            }
+        }
+        named_barrier_sync(1, kConsumerWarps * 32);
+    }
+}
+
+template <int D>
+cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
+                            float *o_part, float *lse_part, cudaStream_t stream) {
+    using Cfg = DecodeCfg<D>;
+    static bool configured[64] = {};
+    const int dev = pool->desc.device & 63;
+    if (!configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(decode_splitk_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             Cfg::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    const float scale_log2 = plan->scale * 1.4426950408889634f;
+    decode_splitk_kernel<D><<<(unsigned)plan->info.decode_ctas, kDecodeThreads, Cfg::kSmemBytes, stream>>>(
+        pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
+        o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, plan->group,
+        pool->desc.num_pages, scale_log2, pool->d_status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int decode_ctas_per_sm(int head_dim) {
+    (void)head_dim;
+    return 1;
+}
+
+cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
+                                 float *lse, float *o_part, float *lse_part, cudaStream_t stream) {
+    if (pool->desc.head_dim == 128) return launch_decode_t<128>(pool, plan, q, out, lse, o_part, lse_part, stream);
+    return launch_decode_t<64>(pool, plan, q, out, lse, o_part, lse_part, stream);
+}
+
+}  // namespace ap

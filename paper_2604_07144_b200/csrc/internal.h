@@ -1,0 +1,131 @@
+// Internal declarations shared by the host code and the kernels of the
+// serving-iteration library.  Not part of the public ABI.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "ap_serving.h"
+
+namespace ap {
+
+constexpr int kPageSize = 16;
+
+// ---- device work lists (all int32, uploaded as one blob per plan) ---------
+
+// One split-K decode work item: the G query heads of one kv head of one decode
+// row over a contiguous range of that sequence's logical pages.
+struct DecodeItem {
+    int32_t q_row;       // row in q / out
+    int32_t kv_head;
+    int32_t bt_offset;   // offset of the sequence's first block-table entry in bt_flat
+    int32_t page_begin;  // first logical page of the range
+    int32_t page_count;  // pages in the range (>= 1)
+    int32_t kv_len;      // attended length of the row (position + 1)
+    int32_t part_slot;   // slot in the partial buffers, or -1: write out/lse directly
+    int32_t pad;
+};
+static_assert(sizeof(DecodeItem) == 32, "DecodeItem layout");
+
+// One (row, kv head) result assembled from several partials.
+struct MergeEntry {
+    int32_t q_row;
+    int32_t kv_head;
+    int32_t part_begin;
+    int32_t part_count;
+};
+
+// One prefill work unit: 128 consecutive query rows of one sequence for one
+// q head, over all keys up to the last row's position.
+struct PrefillTile {
+    int32_t q_row0;      // global row of the tile's first query
+    int32_t rows;        // valid rows in the tile (1..128)
+    int32_t q_head;
+    int32_t kv_head;
+    int32_t bt_offset;
+    int32_t pos0;        // position of the first query row in its sequence
+    int32_t ctx_len;     // sequence context length (positions >= ctx_len hold no token)
+    int32_t pad;
+};
+static_assert(sizeof(PrefillTile) == 32, "PrefillTile layout");
+
+// Partial buffers inside the caller's workspace: o_part [slots][G][d] fp32
+// followed by lse_part [slots][G] fp32.
+struct WorkspaceLayout {
+    size_t o_part_off = 0;
+    size_t lse_part_off = 0;
+    size_t bytes = 0;
+};
+
+// ---- host objects ----------------------------------------------------------
+
+struct PlanBuffer {            // reusable staging for one plan upload
+    int32_t *host = nullptr;   // pinned
+    int32_t *dev = nullptr;
+    size_t capacity = 0;       // int32 elements
+    cudaEvent_t uploaded = nullptr;
+};
+
+}  // namespace ap
+
+struct ap_kv_pool {
+    ap_pool_desc desc{};
+    bool owns_planes = false;
+    int sm_count = 0;
+    int *d_status = nullptr;
+    CUtensorMap k_map{}, v_map{};
+    // allocator
+    std::vector<int32_t> free_list;     // pages handed out from the back
+    std::vector<uint8_t> allocated;     // per page
+    // recycled plan staging
+    std::vector<ap::PlanBuffer> plan_buffers;
+    // staging for ap_serving_iteration_host
+    void *stage_dev = nullptr;
+    size_t stage_bytes = 0;
+};
+
+struct ap_plan {
+    ap_kv_pool *pool = nullptr;
+    ap::PlanBuffer buf{};
+    int num_q_heads = 0;
+    int group = 0;               // G = Hq / Hkv
+    float scale = 0.f;
+    ap_plan_info info{};
+    ap_plan_layout layout{};
+    std::vector<int32_t> blob;   // host copy of the uploaded work lists
+    int n_part_slots = 0;
+    ap::WorkspaceLayout ws{};
+    // device pointers into buf.dev
+    const int32_t *d_append_dst = nullptr;
+    const int32_t *d_bt_flat = nullptr;
+    const ap::DecodeItem *d_items = nullptr;
+    const int32_t *d_cta_begin = nullptr;
+    const ap::MergeEntry *d_merge = nullptr;
+    const ap::PrefillTile *d_tiles = nullptr;
+};
+
+namespace ap {
+
+// Kernel launchers (each returns a cudaError_t from the launch).
+cudaError_t launch_kv_append(const ap_kv_pool *pool, const ap_plan *plan, const void *k_new,
+                             const void *v_new, cudaStream_t stream);
+cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
+                                 float *lse, float *o_part, float *lse_part, cudaStream_t stream);
+cudaError_t launch_lse_merge(const ap_kv_pool *pool, const ap_plan *plan, const float *o_part,
+                             const float *lse_part, void *out, float *lse, cudaStream_t stream);
+cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
+                           float *lse, cudaStream_t stream);
+
+// Decode kernel launch geometry (used by the planner to size the item lists).
+int decode_ctas_per_sm(int head_dim);
+constexpr int kDecodePagesPerStage = 4;
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no libcuda link).
+int encode_pool_tensor_map(CUtensorMap *map, void *base, int num_pages, int num_kv_heads, int head_dim);
+int encode_q_tensor_map(CUtensorMap *map, const void *q, int64_t n_rows, int num_q_heads, int head_dim);
+
+}  // namespace ap

@@ -1,0 +1,123 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Append and page indexing bit-exact; attention
+output within 1e-2 max abs (bf16 out, N(0,1) inputs); lse within 1e-3 relative
+(denominator max(|lse|, 1))."""
+import numpy as np
+import pytest
+
+import paper_2604_07144_b200 as ap
+from paper_2604_07144_b200 import binding as B
+from paper_2604_07144_b200 import workloads as W
+
+from harness import GpuRun, check_batch_full, check_batch_sampled, to_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def decode_batch(seed, shape, ctx_lens, pool_factor=1.3):
+    ctx = np.asarray(ctx_lens, np.int32)
+    return W._assemble(f"decode_{seed}", shape, W.make_rng(seed), np.ones(len(ctx), np.int32), ctx, pool_factor)
+
+
+def test_config1_single_decode_both_readings():
+    for post in (True, False):
+        b = W.config1(post_append=post)
+        err, lerr = check_batch_full(b)
+        print(f"config1 post_append={post}: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def test_decode_page_boundaries_and_tiny_contexts():
+    # first slot of a page, last slot, one token, exactly one stage, one stage + 1 ...
+    ctx = [1, 2, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 1000]
+    check_batch_full(decode_batch(101, W.SHAPE_S1, ctx))
+    check_batch_full(decode_batch(102, W.SHAPE_8B, ctx))
+
+
+@pytest.mark.parametrize("shape", [(8, 8, 64), (8, 4, 64), (6, 2, 128), (32, 8, 128), (64, 8, 128), (5, 1, 128)],
+                         ids=lambda s: f"Hq{s[0]}_Hkv{s[1]}_d{s[2]}")
+def test_decode_head_ratios(shape):
+    rng = np.random.default_rng(7)
+    ctx = rng.integers(1, 700, size=9)
+    check_batch_full(decode_batch(103, shape, ctx))
+
+
+def test_decode_split_and_merge_long_context():
+    # few long sequences: every (row, kv head) stream is cut across many CTAs
+    b = decode_batch(104, W.SHAPE_8B, [20000, 9001, 333])
+    run = GpuRun(b)
+    assert run.info["merge_entries"] > 0 and run.info["decode_ctas"] > 100
+    run.close()
+    check_batch_full(b)
+
+
+def test_decode_explicit_scale():
+    check_batch_full(decode_batch(105, W.SHAPE_S1, [40, 300]), scale=0.05)
+
+
+def test_mixed_ragged_small():
+    for seed in (201, 202, 203):
+        check_batch_full(W.random_ragged(seed, shape=W.SHAPE_S1, batch=7, max_ctx=400, max_q=40))
+    check_batch_full(W.random_ragged(204, shape=W.SHAPE_8B, batch=5, max_ctx=900, max_q=300))
+
+
+def test_prefill_chunk_shapes():
+    # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
+    cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]
+    for i, (ql, cl) in enumerate(cases):
+        b = W._assemble(f"prefill_{i}", W.SHAPE_8B, W.make_rng(300 + i), np.array(ql, np.int32), np.array(cl, np.int32), 1.3)
+        check_batch_full(b)
+
+
+def test_empty_and_skipped_sequences():
+    b = W._assemble("skipped", W.SHAPE_S1, W.make_rng(400), np.array([0, 1, 0], np.int32), np.array([33, 70, 5], np.int32), 1.3)
+    check_batch_full(b)
+    b = W._assemble("all_skipped", W.SHAPE_S1, W.make_rng(401), np.array([0, 0], np.int32), np.array([33, 70], np.int32), 1.3)
+    check_batch_full(b)
+
+
+def test_workspace_too_small_is_reported():
+    b = decode_batch(106, W.SHAPE_8B, [30000])
+    run = GpuRun(b)
+    assert run.workspace_bytes > 0
+    with pytest.raises(ap.ApError) as e:
+        ap.attention_iteration(run.pool, run.plan, run.q, run.out, run.lse, run.workspace, run.workspace_bytes - 1)
+    assert e.value.status == B.AP_ERR_WORKSPACE_TOO_SMALL
+    run.close()
+
+
+def test_config2_full_size_sampled():
+    err, lerr = check_batch_sampled(W.config2(), n_samples=256)
+    print(f"config2: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def test_config3_full_size_sampled():
+    err, lerr = check_batch_sampled(W.config3(), n_samples=256)
+    print(f"config3: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def test_config4_full_size_sampled():
+    err, lerr = check_batch_sampled(W.config4(), n_samples=48)
+    print(f"config4: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def test_host_buffer_iteration_matches_device_path():
+    import torch
+    b = W.random_ragged(501, shape=W.SHAPE_8B, batch=6, max_ctx=500, max_q=1)
+    b.q_lens[:] = 1
+    b = decode_batch(502, W.SHAPE_8B, [77, 500, 1300, 16])
+    run = GpuRun(b)
+    run.append(); run.attend()
+    assert run.status() == 0
+    ref_out, ref_lse = to_bits(run.out)[:b.n_new].copy(), run.lse.cpu().numpy()[:b.n_new].copy()
+    ref_k = to_bits(run.k_pool).copy()
+    run.close()
+    run = GpuRun(b)                                  # fresh pool (pre-append state)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+    q, kn, vn = pin(b.q), pin(b.k_new), pin(b.v_new)
+    out = torch.empty((b.n_new, b.num_q_heads, b.head_dim), dtype=torch.int16).pin_memory()
+    lse = torch.empty((b.n_new, b.num_q_heads), dtype=torch.float32).pin_memory()
+    ap.serving_iteration_host(run.pool, b.q_lens, b.ctx_lens, b.block_tables, b.num_q_heads, q, kn, vn, out, lse)
+    assert np.array_equal(out.numpy().view(np.uint16), ref_out)
+    assert np.array_equal(lse.numpy(), ref_lse)
+    assert np.array_equal(to_bits(run.k_pool), ref_k)
+    run.close()

@@ -1,0 +1,215 @@
+"""Host logic of the library on a host-only pool (no GPU): page allocator,
+batch validation, and coverage of the planner's work lists."""
+import numpy as np
+import pytest
+
+import paper_2604_07144_b200 as ap
+from paper_2604_07144_b200 import binding as B
+from paper_2604_07144_b200 import workloads as W
+
+
+def host_pool(num_pages=64, hkv=2, d=64):
+    return ap.kv_pool_create(num_pages, hkv, d, device=-1)
+
+
+def test_pool_create_rejects_bad_descriptions():
+    for kw in (dict(num_pages=0, num_kv_heads=2, head_dim=64), dict(num_pages=4, num_kv_heads=0, head_dim=64)):
+        with pytest.raises(ap.ApError) as e:
+            ap.kv_pool_create(device=-1, **kw)
+        assert e.value.status == B.AP_ERR_INVALID_ARG
+    for kw in (dict(head_dim=96), dict(head_dim=64, page_size=32)):
+        with pytest.raises(ap.ApError) as e:
+            ap.kv_pool_create(4, 2, device=-1, **kw)
+        assert e.value.status == B.AP_ERR_UNSUPPORTED
+
+
+def test_allocator_all_or_nothing_and_double_free():
+    pool = host_pool(10)
+    a = ap.kv_pool_alloc_pages(pool, 4)
+    assert list(a) == [0, 1, 2, 3] and ap.kv_pool_num_free(pool) == 6
+    with pytest.raises(ap.ApError) as e:
+        ap.kv_pool_alloc_pages(pool, 7)
+    assert e.value.status == B.AP_ERR_OUT_OF_PAGES and ap.kv_pool_num_free(pool) == 6
+    b = ap.kv_pool_alloc_pages(pool, 6)
+    assert sorted(list(a) + list(b)) == list(range(10))
+    ap.kv_pool_free_pages(pool, a[:2])
+    for bad in ([int(a[0])], [int(a[2]), int(a[2])], [10], [-1]):
+        with pytest.raises(ap.ApError) as e:
+            ap.kv_pool_free_pages(pool, bad)
+        assert e.value.status == B.AP_ERR_INVALID_ARG
+    assert ap.kv_pool_num_free(pool) == 2
+    ap.kv_pool_free_pages(pool, [int(a[2])])     # the rejected calls freed nothing
+    assert sorted(ap.kv_pool_alloc_pages(pool, 3)) == sorted(int(x) for x in a[:3])
+    ap.kv_pool_destroy(pool)
+
+
+def test_seeded_free_list_is_a_permutation_and_deterministic():
+    orders = []
+    for _ in range(2):
+        pool = host_pool(100)
+        ap.kv_pool_seed_free_list(pool, 1234)
+        orders.append(list(ap.kv_pool_alloc_pages(pool, 100)))
+        ap.kv_pool_destroy(pool)
+    assert orders[0] == orders[1]
+    assert sorted(orders[0]) == list(range(100)) and orders[0] != list(range(100))
+
+
+def test_plan_validation():
+    pool = host_pool(8)
+    bt = np.array([[0, 1, 2, -1]], np.int32)
+    ok = ap.plan_create(pool, [1], [33], bt, 8)
+    assert ap.plan_get_info(ok)["n_new"] == 1
+    ap.plan_destroy(ok)
+    cases = [
+        (([2], [1], bt, 8), B.AP_ERR_INVALID_ARG),            # q_len > ctx_len
+        (([-1], [5], bt, 8), B.AP_ERR_INVALID_ARG),
+        (([1], [65], bt, 8), B.AP_ERR_INVALID_ARG),           # table too short
+        (([1], [49], bt, 8), B.AP_ERR_BAD_BLOCK_TABLE),       # reaches the -1 entry
+        (([1], [33], np.array([[0, 1, 8, 0]], np.int32), 8), B.AP_ERR_BAD_BLOCK_TABLE),  # page id == num_pages
+        (([1], [33], bt, 7), B.AP_ERR_INVALID_ARG),           # heads not a multiple
+        (([1], [33], bt, 32), B.AP_ERR_UNSUPPORTED),          # group of 16
+    ]
+    for args, status in cases:
+        with pytest.raises(ap.ApError) as e:
+            ap.plan_create(pool, *args)
+        assert e.value.status == status, args
+    # two sequences appending into the same slot
+    bt2 = np.array([[3, -1], [3, -1]], np.int32)
+    with pytest.raises(ap.ApError) as e:
+        ap.plan_create(pool, [1, 1], [5, 5], bt2, 8)
+    assert e.value.status == B.AP_ERR_BAD_BLOCK_TABLE
+    # sharing a page for reading only is legal
+    bt3 = np.array([[3, 4], [3, 5]], np.int32)
+    ap.plan_destroy(ap.plan_create(pool, [1, 1], [17, 17], bt3, 8))
+    # q_len 0 sequences are skipped, even with garbage tables
+    p = ap.plan_create(pool, [0, 1], [40, 17], np.array([[-5, -5, -5], [3, 4, -1]], np.int32), 8)
+    assert ap.plan_get_info(p)["kv_tokens"] == 17
+    ap.plan_destroy(p)
+    # a host-only pool cannot launch
+    p = ap.plan_create(pool, [1], [33], bt, 8)
+    with pytest.raises(ap.ApError) as e:
+        ap.kv_append(pool, p, 0, 0)
+    assert e.value.status == B.AP_ERR_CUDA
+    ap.plan_destroy(p)
+    ap.kv_pool_destroy(pool)
+
+
+def check_plan_coverage(batch: W.Batch):
+    """Every (decode row, kv head, page) appears in exactly one item; merge
+    entries and part slots are consistent; every prefill row/head is in one tile."""
+    hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
+    pool = ap.kv_pool_create(batch.num_pages, hkv, d, device=-1)
+    plan = ap.plan_create(pool, batch.q_lens, batch.ctx_lens, batch.block_tables, hq)
+    ex = ap.plan_export(plan)
+    info = ex["info"]
+    rows = batch.q_indptr
+    assert info["n_new"] == batch.n_new and info["kv_tokens"] == batch.kv_tokens
+    # append destinations
+    exp = []
+    for s in range(batch.batch):
+        for t in range(int(batch.q_lens[s])):
+            p = int(batch.ctx_lens[s]) - int(batch.q_lens[s]) + t
+            exp.append(int(batch.block_tables[s, p // 16]) * 16 + p % 16)
+    assert list(ex["append_dst"]) == exp
+    # decode coverage
+    items, cta = ex["decode_items"], ex["cta_begin"]
+    seen = {}
+    row_to_seq = {int(rows[s]): s for s in range(batch.batch) if batch.q_lens[s] == 1}
+    for q_row, kvh, bt_off, pb, pc, kv_len, slot, _ in items:
+        s = row_to_seq[int(q_row)]
+        assert kv_len == batch.ctx_lens[s] and pc >= 1 and 0 <= kvh < hkv
+        npages = (int(batch.ctx_lens[s]) + 15) // 16
+        assert 0 <= pb and pb + pc <= npages
+        if pb + pc < npages:
+            assert pc % 4 == 0                      # cuts fall on stage boundaries
+        assert list(ex["bt_flat"][bt_off:bt_off + npages]) == list(batch.block_tables[s, :npages])
+        for pg in range(pb, pb + pc):
+            assert (s, int(kvh), pg) not in seen
+            seen[(s, int(kvh), pg)] = int(slot)
+    want = {(s, g, pg) for s in row_to_seq.values() for g in range(hkv)
+            for pg in range((int(batch.ctx_lens[s]) + 15) // 16)}
+    assert set(seen) == want
+    if len(items):
+        assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) > 0).all()
+        assert len(cta) - 1 == info["decode_ctas"] <= 148
+        cost = [int(items[a:b, 4].sum()) for a, b in zip(cta[:-1], cta[1:])]
+        if sum(cost) >= 148 * 64:                   # enough work to balance
+            assert max(cost) <= 1.15 * (sum(cost) / len(cost)) + 8
+    # merge entries
+    slots = sorted(int(x) for x in items[:, 6] if x >= 0) if len(items) else []
+    assert slots == list(range(len(slots)))
+    covered = []
+    for q_row, kvh, pb, pc in ex["merge_entries"]:
+        assert pc >= 2
+        its = items[(items[:, 0] == q_row) & (items[:, 1] == kvh)]
+        assert sorted(int(x) for x in its[:, 6]) == list(range(pb, pb + pc))
+        covered += list(range(pb, pb + pc))
+    assert sorted(covered) == slots
+    single = items[items[:, 6] < 0] if len(items) else items
+    for it in single:
+        assert it[3] == 0 and it[4] == (int(it[5]) + 15) // 16
+    # prefill coverage
+    seen_rows = set()
+    for q_row0, nrows, qh, kvh, bt_off, pos0, ctx, _ in ex["prefill_tiles"]:
+        assert 1 <= nrows <= 128 and kvh == qh // (hq // hkv)
+        for r in range(q_row0, q_row0 + nrows):
+            assert (r, int(qh)) not in seen_rows
+            seen_rows.add((r, int(qh)))
+        s = int(np.searchsorted(rows, q_row0, side="right") - 1)
+        assert ctx == batch.ctx_lens[s] and pos0 == ctx - batch.q_lens[s] + (q_row0 - rows[s])
+    want_rows = {(r, h) for s in range(batch.batch) if batch.q_lens[s] > 1
+                 for r in range(int(rows[s]), int(rows[s + 1])) for h in range(hq)}
+    assert seen_rows == want_rows
+    ends = [int(t[5] + t[1]) for t in ex["prefill_tiles"]]
+    assert ends == sorted(ends, reverse=True)        # longest first
+    ap.plan_destroy(plan)
+    ap.kv_pool_destroy(pool)
+    return info
+
+
+def test_plan_coverage_small_and_ragged():
+    for seed in range(20, 30):
+        check_plan_coverage(W.random_ragged(seed, batch=9, max_ctx=700, max_q=3))
+    check_plan_coverage(W.config1())
+    info = check_plan_coverage(W.random_ragged(5, batch=6, max_ctx=900, max_q=300))
+    assert info["prefill_tiles"] > 0
+
+
+def test_plan_coverage_full_size_configs():
+    i2 = check_plan_coverage(W.config2(with_pool=False))
+    assert i2["decode_rows"] == 64 and i2["decode_ctas"] == 148
+    i3 = check_plan_coverage(W.config3(with_pool=False))
+    assert i3["prefill_seqs"] == 8 and i3["decode_rows"] == 120 and i3["prefill_tiles"] == 8 * 4 * 32
+    i4 = check_plan_coverage(W.config4(with_pool=False))
+    assert i4["decode_ctas"] == 148 and i4["merge_entries"] > 0
+
+
+def test_empty_batch_plans_to_nothing():
+    pool = host_pool()
+    p = ap.plan_create(pool, [], [], np.zeros((0, 1), np.int32), 8)
+    info = ap.plan_get_info(p)
+    assert info["n_new"] == 0 and info["launches_attention"] == 0 and ap.plan_workspace_bytes(p) == 0
+    ap.plan_destroy(p)
+    ap.kv_pool_destroy(pool)
+
+
+def test_trace_generator_invariants():
+    reqs = W.trace_arrivals(iterations=120)
+    peak = W.trace_peak_pages(reqs, iterations=120)
+    alloc = W.FreeListAllocator(int(1.25 * peak) + 1)
+    owner = {}
+    done_tokens = 0
+    for it in W.fcfs_trace(reqs, alloc.alloc, alloc.free, iterations=120):
+        assert int(it.q_lens.sum()) <= 8192
+        assert (it.q_lens >= 1).all() and (it.q_lens <= 512).all() and (it.ctx_lens >= it.q_lens).all()
+        pf = it.q_lens > 1
+        assert not pf[np.argmax(~pf):].any() if (~pf).any() else True     # prefill rows first
+        used = set()
+        for i, rid in enumerate(it.rids):
+            n = (int(it.ctx_lens[i]) + 15) // 16
+            pages = [int(p) for p in it.block_tables[i, :n]]
+            assert all(p >= 0 for p in pages) and not (used & set(pages))
+            used |= set(pages)
+            assert owner.setdefault(int(rid), pages[:len(owner.get(int(rid), []))] or pages)[:1] == pages[:1]
+        done_tokens += int(it.q_lens.sum())
+    assert done_tokens > 0 and alloc.peak_used <= peak
