@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KV serving iteration (KV append + GQA attention).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2|3|4]
+
+A step is one pass of the whole hot path over one synthetic batch: KV append,
+split-K decode attention, LSE merge and (for batches with prefill chunks)
+prefill attention.  The default workload is the decode-heavy ragged batch on
+the Llama-3-8B attention shape (64 sequences, contexts log-uniform in
+128..8192).  Prints ONE JSON line (rank 0).
+
+Timing: CUDA events on the launching stream around exactly K steps after W
+warm-up steps, barrier + synchronize on both sides, max over ranks.  Every
+step reads a different copy of the KV pool (rotation among copies whose
+combined size is many times the L2), so KV reads are cold.  The plan (host
+work list + one H2D copy) is built once per batch outside `value`'s timed
+region -- a serving engine builds it once per iteration and reuses it for
+every layer -- and is inside the `e2e` region, which goes through
+ap_serving_iteration_host with pinned host buffers every step.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "serving_iteration_attention_kv_tokens_per_s"
+UNIT = "KV-tokens/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitk launch on the
+# bench workload (ncu capture summarised under profiles/), keyed by the hash of
+# the kernel source the counters were taken from; a changed kernel reports null.
+NCU_TRAFFIC = {}
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for f in ("decode_splitk.cu", "ptx.cuh", "internal.h"):
+        with open(os.path.join(ROOT, "paper_2604_07144_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def make_batch(config: int, seed_offset: int = 0, with_pool: bool = True):
+    from paper_2604_07144_b200 import workloads as W
+    gen = {1: W.config1, 2: W.config2, 3: W.config3, 4: W.config4}[config]
+    kw = {} if config == 1 else {"with_pool": with_pool}
+    return gen(seed=W.SEED_BASE + config + 1000 * seed_offset, **kw)
+
+
+def algorithmic_bytes(batch, info):
+    """Bytes the method must move per step (one attention layer)."""
+    hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
+    per_kv_token = 2 * hkv * d * 2
+    per_row = 2 * hq * d * 2 + hq * 4                      # q read, out write, lse write
+    dec = batch.q_lens == 1
+    decode_kv = int(batch.ctx_lens[dec].astype(np.int64).sum())
+    decode_bytes = decode_kv * per_kv_token + int(dec.sum()) * per_row + int(((batch.ctx_lens[dec] + 15) // 16).sum()) * 4
+    append_bytes = 2 * info["n_new"] * 2 * hkv * d * 2     # read + write, K and V
+    total = info["kv_tokens"] * per_kv_token + info["n_new"] * per_row + append_bytes
+    return {"per_kv_token": per_kv_token, "decode_kernel": decode_bytes, "total": total}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def cpu_oracle_baseline(batch, target_s: float = 12.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of
+    the same workload: whole sequences of the batch, in batch order, until the
+    estimated time reaches target_s (first a one-sequence probe)."""
+    import oracle
+    oracle.lib()
+    k, v = batch.k_pool.copy(), batch.v_pool.copy()
+    oracle.kv_append(k, v, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.k_new, batch.v_new)
+    rows = batch.q_indptr
+
+    def run(seqs):
+        ql = np.zeros_like(batch.q_lens)
+        ql[seqs] = batch.q_lens[seqs]
+        qsel = np.concatenate([batch.q[rows[s]:rows[s + 1]] for s in seqs])
+        t0 = time.perf_counter()
+        oracle.attention(k, v, ql, batch.ctx_lens, batch.block_tables, qsel)
+        return time.perf_counter() - t0, int(batch.ctx_lens[seqs].astype(np.int64).sum())
+
+    active = [int(s) for s in np.nonzero(batch.q_lens > 0)[0]]
+    # cost of a sequence ~ q_len * ctx_len
+    cost = {s: float(batch.q_lens[s]) * float(batch.ctx_lens[s]) for s in active}
+    probe = min(active, key=lambda s: cost[s])
+    t_probe, _ = run([probe])
+    rate = cost[probe] / max(t_probe, 1e-6)
+    chosen, est = [], 0.0
+    for s in active:
+        if chosen and est + cost[s] / rate > target_s:
+            continue
+        chosen.append(s)
+        est += cost[s] / rate
+    t, toks = run(chosen)
+    return {"value": toks / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(chosen)} of {len(active)} sequences of the workload ({toks} KV-tokens, "
+                      f"all heads, fp64, {t:.2f} s)"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    batch = make_batch(args.config)
+    oracle.lib()
+    k, v = batch.k_pool.copy(), batch.v_pool.copy()
+    rows = batch.q_indptr
+    active = [int(s) for s in np.nonzero(batch.q_lens > 0)[0]]
+    # bounded sample: the sequences with the smallest q_len*ctx_len cost first, ~2 s per step
+    t0 = time.perf_counter()
+    oracle.kv_append(k, v, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.k_new, batch.v_new)
+    s0 = min(active, key=lambda s: float(batch.q_lens[s]) * float(batch.ctx_lens[s]))
+    ql = np.zeros_like(batch.q_lens); ql[s0] = batch.q_lens[s0]
+    t1 = time.perf_counter()
+    oracle.attention(k, v, ql, batch.ctx_lens, batch.block_tables, batch.q[rows[s0]:rows[s0 + 1]])
+    rate = float(batch.q_lens[s0]) * float(batch.ctx_lens[s0]) / max(time.perf_counter() - t1, 1e-6)
+    chosen, est = [], 0.0
+    for s in active:
+        c = float(batch.q_lens[s]) * float(batch.ctx_lens[s]) / rate
+        if chosen and est + c > 2.0:
+            continue
+        chosen.append(s); est += c
+    ql = np.zeros_like(batch.q_lens); ql[chosen] = batch.q_lens[chosen]
+    qsel = np.concatenate([batch.q[rows[s]:rows[s + 1]] for s in chosen])
+    knew = np.concatenate([batch.k_new[rows[s]:rows[s + 1]] for s in chosen])
+    vnew = np.concatenate([batch.v_new[rows[s]:rows[s + 1]] for s in chosen])
+    toks = int(batch.ctx_lens[chosen].astype(np.int64).sum())
+
+    def step():
+        oracle.kv_append(k, v, ql, batch.ctx_lens, batch.block_tables, knew, vnew)
+        oracle.attention(k, v, ql, batch.ctx_lens, batch.block_tables, qsel)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = toks * args.steps / dt
+    sample = f"{len(chosen)} of {len(active)} sequences of the workload per step ({toks} KV-tokens, all heads, fp64)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": batch.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap_ = argparse.ArgumentParser()
+    ap_.add_argument("--gpus", type=int, default=1)
+    ap_.add_argument("--steps", type=int, default=300)
+    ap_.add_argument("--warmup", type=int, default=10)
+    ap_.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap_.add_argument("--config", type=int, default=2, choices=[2, 3, 4])
+    ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
+    ap_.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap_.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2604_07144_b200 as ap
+    from paper_2604_07144_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # replicas only: every rank serves its own independent batch, no data-path collective
+    batch = make_batch(args.config, seed_offset=rank)
+    hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
+
+    def dev_bf16(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    kv_bytes = batch.kv_tokens * 2 * hkv * d * 2
+    copies = args.pool_copies or max(3, int(np.ceil(2.0e9 / max(kv_bytes, 1))))
+    copies = min(copies, 16)
+    pools, plans, k_planes, v_planes = [], [], [], []
+    k0, v0 = dev_bf16(batch.k_pool), dev_bf16(batch.v_pool)
+    for c in range(copies):
+        kp, vp = (k0, v0) if c == 0 else (k0.clone(), v0.clone())
+        k_planes.append(kp); v_planes.append(vp)
+        pools.append(ap.kv_pool_create(batch.num_pages, hkv, d, kp, vp, device=local_rank))
+        plans.append(ap.plan_create(pools[-1], batch.q_lens, batch.ctx_lens, batch.block_tables, hq))
+    info = ap.plan_get_info(plans[0])
+    q, k_new, v_new = dev_bf16(batch.q), dev_bf16(batch.k_new), dev_bf16(batch.v_new)
+    out = torch.empty((batch.n_new, hq, d), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((batch.n_new, hq), dtype=torch.float32, device=dev)
+    ws_bytes = ap.plan_workspace_bytes(plans[0])
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+
+    def step(i):
+        c = i % copies
+        ap.kv_append(pools[c], plans[c], k_new, v_new)
+        ap.attention_iteration(pools[c], plans[c], q, out, lse, ws, ws_bytes)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def reduce_max(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def reduce_sum(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    # ---- device-resident timing
+    for i in range(args.warmup):
+        step(i)
+    for p in pools:
+        assert ap.last_device_status(p) == 0
+        ap.profile_enable(p, True)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_total = reduce_max(e0.elapsed_time(e1))
+    clocks = sampler.stop() if rank == 0 else None
+    kt = {}
+    for p in pools:
+        for name, (ms, n) in ap.profile_collect(p).items():
+            a = kt.setdefault(name, [0.0, 0])
+            a[0] += ms; a[1] += n
+        ap.profile_enable(p, False)
+        assert ap.last_device_status(p) == 0
+    total_tokens = reduce_sum(float(batch.kv_tokens))
+    ms_per_step = ms_total / args.steps
+    value = total_tokens / (ms_per_step * 1e-3)
+
+    # ---- plan cost (host + upload), reported separately
+    t0 = time.perf_counter()
+    for _ in range(20):
+        ap.plan_destroy(ap.plan_create(pools[0], batch.q_lens, batch.ctx_lens, batch.block_tables, hq))
+    torch.cuda.synchronize()
+    plan_ms = (time.perf_counter() - t0) / 20 * 1e3
+
+    # ---- end to end through the host-buffer entry point
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+    hq_, hk_, hv_ = pin(batch.q), pin(batch.k_new), pin(batch.v_new)
+    hout = torch.empty((batch.n_new, hq, d), dtype=torch.int16).pin_memory()
+    hlse = torch.empty((batch.n_new, hq), dtype=torch.float32).pin_memory()
+
+    def e2e_step(i):
+        ap.serving_iteration_host(pools[i % copies], batch.q_lens, batch.ctx_lens, batch.block_tables, hq,
+                                  hq_, hk_, hv_, hout, hlse)
+
+    e2e_steps = max(10, args.steps // 4)
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_ms = reduce_max(e0.elapsed_time(e1)) / e2e_steps
+    h2d = int(batch.q.nbytes + batch.k_new.nbytes + batch.v_new.nbytes)
+    d2h = int(hout.numel() * 2 + hlse.numel() * 4)
+
+    # sanity: the timed path produced finite numbers
+    assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
+
+    if rank == 0:
+        peaks = measured_peaks()
+        alg = algorithmic_bytes(batch, info)
+        dec_ms, dec_n = kt.get("decode_splitk", (0.0, 0))
+        # the profile sums cover this rank's launches only
+        achieved = alg["decode_kernel"] / (dec_ms / max(dec_n, 1) * 1e-3) / 1e9 if dec_n else 0.0
+        roofline = {
+            "bound": "hbm", "kernel": "decode_splitk", "achieved": achieved, "peak": peaks["hbm_gbs"],
+            "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+            "traffic": NCU_TRAFFIC.get((args.config, kernel_source_hash())),
+            "bytes_per_launch": alg["decode_kernel"], "us_per_launch": 1e3 * dec_ms / max(dec_n, 1),
+            "frac_of_nominal_8TBs": achieved / 8000.0,
+        }
+        kernels = {name: {"launches": n, "us_per_launch": (1e3 * ms / n if n else None)} for name, (ms, n) in kt.items()}
+        res = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": batch.name, "num_q_heads": hq, "num_kv_heads": hkv, "head_dim": d,
+                       "page_size": 16, "sequences": batch.batch, "new_tokens": batch.n_new,
+                       "kv_tokens_per_step_per_gpu": batch.kv_tokens,
+                       "l2": f"rotation among {copies} pool copies ({copies * kv_bytes / 1e9:.2f} GB of KV, each step's "
+                             f"{kv_bytes / 1e6:.0f} MB larger than the 126 MB L2)",
+                       "parallelism": "replicas only (one independent batch per GPU, no collective)"},
+            "gpu_launches": int(sum(n for _, n in kt.values())),
+            "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                    "includes": "plan build + upload, H2D of q/k_new/v_new, append, attention, D2H of out/lse, sync"},
+            "plan": {"host_ms": plan_ms, "in_value": False, "in_e2e": True, **{k: info[k] for k in (
+                "decode_items", "decode_ctas", "merge_entries", "prefill_tiles")}},
+            "roofline": roofline,
+            "kernels": kernels,
+            "step_gbs": alg["total"] / (ms_per_step * 1e-3) / 1e9,
+            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            res["cpu_baseline"] = cpu_oracle_baseline(batch)
+        print(json.dumps(res))
+
+    for pl in plans:
+        ap.plan_destroy(pl)
+    for p in pools:
+        ap.kv_pool_destroy(p)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -219,6 +219,23 @@ int ap_last_device_status(ap_kv_pool *pool, void *stream);
 
 const char *ap_status_string(int status);
 
+/* ----------------------------------------------------------- diagnostics -- */
+
+/*
+ * Per-kernel device timing for benchmarks.  While enabled, every kernel the
+ * library launches for this pool is bracketed by CUDA events recorded on the
+ * launching stream.  ap_profile_collect synchronises `stream`, adds up the
+ * elapsed times per kernel since the last enable/collect, and clears the
+ * records.  Index: 0 kv_append, 1 decode split-K, 2 LSE merge, 3 prefill.
+ */
+enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_MERGE = 2, AP_KERNEL_PREFILL = 3, AP_KERNEL_COUNT = 4 };
+typedef struct ap_kernel_times {
+    double ms[AP_KERNEL_COUNT];
+    int64_t launches[AP_KERNEL_COUNT];
+} ap_kernel_times;
+int ap_profile_enable(ap_kv_pool *pool, int on);
+int ap_profile_collect(ap_kv_pool *pool, void *stream, ap_kernel_times *out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -36,6 +36,7 @@ EXPORTED_SYMBOLS = (
     "ap_kv_pool_seed_free_list", "ap_kv_pool_num_free", "ap_plan_create", "ap_plan_destroy",
     "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append",
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
+    "ap_profile_enable", "ap_profile_collect",
 )
 
 
@@ -73,6 +74,12 @@ class PlanLayout(ctypes.Structure):
         "prefill_tiles", "n_bt", "n_cta_begin")]
 
 
+class KernelTimes(ctypes.Structure):
+    _fields_ = [("ms", ctypes.c_double * 4), ("launches", ctypes.c_int64 * 4)]
+
+
+KERNEL_NAMES = ("kv_append", "decode_splitk", "lse_merge", "prefill")
+
 _lib: Optional[ctypes.CDLL] = None
 
 
@@ -108,6 +115,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_attention_iteration": (ctypes.c_int, [vp, vp, vp, vp, vp, vp, sz, vp]),
         "ap_serving_iteration_host": (ctypes.c_int, [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, vp]),
         "ap_last_device_status": (ctypes.c_int, [vp, vp]),
+        "ap_profile_enable": (ctypes.c_int, [vp, ctypes.c_int]),
+        "ap_profile_collect": (ctypes.c_int, [vp, vp, ctypes.POINTER(KernelTimes)]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -316,3 +325,16 @@ def serving_iteration_host(pool: KVPool, q_lens, ctx_lens, block_tables, num_q_h
 
 def last_device_status(pool: KVPool, stream=None) -> int:
     return int(load().ap_last_device_status(pool.handle, _stream(stream)))
+
+
+# ------------------------------------------------------------ diagnostics --
+
+def profile_enable(pool: KVPool, on: bool = True) -> None:
+    _check(load().ap_profile_enable(pool.handle, int(bool(on))), "ap_profile_enable")
+
+
+def profile_collect(pool: KVPool, stream=None) -> dict:
+    """{kernel name: (total ms, launches)} since the last enable/collect."""
+    kt = KernelTimes()
+    _check(load().ap_profile_collect(pool.handle, _stream(stream), ctypes.byref(kt)), "ap_profile_collect")
+    return {name: (float(kt.ms[i]), int(kt.launches[i])) for i, name in enumerate(KERNEL_NAMES)}

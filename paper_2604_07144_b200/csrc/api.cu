@@ -73,6 +73,36 @@ int acquire_plan_buffer(ap_kv_pool *pool, size_t n_ints, PlanBuffer *out) {
     return AP_OK;
 }
 
+cudaEvent_t take_event(ap_kv_pool *pool) {
+    if (!pool->spare_events.empty()) {
+        cudaEvent_t e = pool->spare_events.back();
+        pool->spare_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreate(&e) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return e;
+}
+
+// Brackets one kernel launch with events when profiling is on.
+struct TimedScope {
+    ap_kv_pool *pool;
+    cudaStream_t stream;
+    TimedLaunch rec{};
+    bool on = false;
+    TimedScope(ap_kv_pool *p, int kernel, cudaStream_t st) : pool(p), stream(st) {
+        if (!p->profiling) return;
+        rec.kernel = kernel;
+        rec.start = take_event(p);
+        rec.stop = take_event(p);
+        on = rec.start && rec.stop && cudaEventRecord(rec.start, st) == cudaSuccess;
+    }
+    ~TimedScope() {
+        if (!on) return;
+        if (cudaEventRecord(rec.stop, stream) == cudaSuccess) pool->timed.push_back(rec);
+    }
+};
+
 }  // namespace
 
 extern "C" {
@@ -173,6 +203,8 @@ int ap_kv_pool_destroy(ap_kv_pool *pool) {
     DeviceGuard guard(pool->desc.device);
     if (guard.ok) (void)cudaDeviceSynchronize();
     for (auto &b : pool->plan_buffers) release_plan_buffer(b);
+    for (auto &t : pool->timed) { (void)cudaEventDestroy(t.start); (void)cudaEventDestroy(t.stop); }
+    for (auto &e : pool->spare_events) (void)cudaEventDestroy(e);
     if (pool->stage_dev) (void)cudaFree(pool->stage_dev);
     if (pool->d_status) (void)cudaFree(pool->d_status);
     if (pool->owns_planes) {
@@ -496,6 +528,7 @@ int ap_kv_append(ap_kv_pool *pool, const ap_plan *plan, const void *k_new, const
     if (!k_new || !v_new || (((uintptr_t)k_new | (uintptr_t)v_new) & 15u)) return AP_ERR_INVALID_ARG;
     DeviceGuard guard(pool->desc.device);
     if (!guard.ok) return AP_ERR_CUDA;
+    TimedScope timed(pool, AP_KERNEL_APPEND, (cudaStream_t)stream);
     if (launch_kv_append(pool, plan, k_new, v_new, (cudaStream_t)stream) != cudaSuccess) {
         (void)cudaGetLastError();
         return AP_ERR_CUDA;
@@ -519,10 +552,18 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
     float *o_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.o_part_off) : nullptr;
     float *lse_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.lse_part_off) : nullptr;
     cudaError_t e = cudaSuccess;
-    if (plan->info.decode_items > 0) e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-    if (e == cudaSuccess && plan->info.merge_entries > 0)
+    if (plan->info.decode_items > 0) {
+        TimedScope timed(pool, AP_KERNEL_DECODE, st);
+        e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+    }
+    if (e == cudaSuccess && plan->info.merge_entries > 0) {
+        TimedScope timed(pool, AP_KERNEL_MERGE, st);
         e = launch_lse_merge(pool, plan, o_part, lse_part, out, lse, st);
-    if (e == cudaSuccess && plan->info.prefill_tiles > 0) e = launch_prefill(pool, plan, q, out, lse, st);
+    }
+    if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
+        TimedScope timed(pool, AP_KERNEL_PREFILL, st);
+        e = launch_prefill(pool, plan, q, out, lse, st);
+    }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return e == cudaErrorNotSupported ? AP_ERR_UNSUPPORTED : AP_ERR_CUDA;
@@ -550,6 +591,42 @@ int ap_last_device_status(ap_kv_pool *pool, void *stream) {
         }
     }
     return status;
+}
+
+int ap_profile_enable(ap_kv_pool *pool, int on) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    for (auto &t : pool->timed) {
+        pool->spare_events.push_back(t.start);
+        pool->spare_events.push_back(t.stop);
+    }
+    pool->timed.clear();
+    pool->profiling = on != 0;
+    return AP_OK;
+}
+
+int ap_profile_collect(ap_kv_pool *pool, void *stream, ap_kernel_times *out) {
+    if (!pool || !out) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    std::memset(out, 0, sizeof(*out));
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) { (void)cudaGetLastError(); return AP_ERR_CUDA; }
+    int rc = AP_OK;
+    for (auto &t : pool->timed) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.start, t.stop) == cudaSuccess && t.kernel >= 0 && t.kernel < AP_KERNEL_COUNT) {
+            out->ms[t.kernel] += ms;
+            out->launches[t.kernel] += 1;
+        } else {
+            (void)cudaGetLastError();
+            rc = AP_ERR_CUDA;
+        }
+        pool->spare_events.push_back(t.start);
+        pool->spare_events.push_back(t.stop);
+    }
+    pool->timed.clear();
+    return rc;
 }
 
 int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, const void *q_host,

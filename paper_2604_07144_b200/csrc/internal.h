@@ -70,6 +70,11 @@ struct PlanBuffer {            // reusable staging for one plan upload
     cudaEvent_t uploaded = nullptr;
 };
 
+struct TimedLaunch {
+    int kernel;
+    cudaEvent_t start, stop;
+};
+
 }  // namespace ap
 
 struct ap_kv_pool {
@@ -86,6 +91,10 @@ struct ap_kv_pool {
     // staging for ap_serving_iteration_host
     void *stage_dev = nullptr;
     size_t stage_bytes = 0;
+    // per-kernel event timing (diagnostics)
+    bool profiling = false;
+    std::vector<ap::TimedLaunch> timed;
+    std::vector<cudaEvent_t> spare_events;
 };
 
 struct ap_plan {
