@@ -202,6 +202,46 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
                            float *lse, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Attention without any device-memory allocation.  (The paper has no
+ * counterpart to this call; it exists for integration reasons only.)
+ *
+ * Who needs it: code that is not allowed to call cudaMalloc at the point where
+ * attention runs -- a serving loop whose memory is entirely owned by a
+ * framework's caching allocator (a raw cudaMalloc can then fail even though
+ * memory is "free"), a latency-critical path that cannot take cudaMalloc's
+ * device-wide synchronisation, or a plug-in that is handed tensors but no
+ * allocator.  Such callers have nowhere to get the split-K workspace that
+ * ap_attention_iteration asks for.
+ *
+ * This variant does the same work as ap_attention_iteration but keeps the
+ * split-K partials in a fixed array of AP_STATIC_WORKSPACE_BYTES (4 MiB) that
+ * is part of the library image: every GPU context that loads the library
+ * holds those 4 MiB until the process exits, used or not.  The call itself
+ * performs no cudaMalloc / cudaFree and calls no allocating routine; q, out
+ * and lse are still the caller's.  (Building the plan is a separate, earlier
+ * call; ap_plan_create recycles its upload buffers and only allocates when it
+ * needs a larger one than it has seen before.)
+ *
+ *  - A plan whose ap_plan_workspace_bytes() exceeds AP_STATIC_WORKSPACE_BYTES
+ *    is rejected with AP_ERR_WORKSPACE_TOO_SMALL before anything is launched
+ *    (4 MiB covers every plan the planner makes for 148 SMs at head_dim 128
+ *    and 8 query heads per kv head, including 131072-token contexts).
+ *  - The first call on each device looks up the array's device address (one
+ *    runtime query, cached afterwards); make that first call outside any
+ *    stream capture.
+ *  - All calls on a device share the one array, and it keeps whatever the last
+ *    call left in it.  Nothing has to start at zero: every partial is written
+ *    in full before it is read within the same call.  Two calls that overlap
+ *    on the GPU (different streams, no ordering between them) race on the
+ *    array and produce garbage; order them, or use ap_attention_iteration with
+ *    separate workspaces.
+ */
+#define AP_STATIC_WORKSPACE_BYTES (4u << 20)
+size_t ap_static_workspace_bytes(void);
+int ap_attention_iteration_static(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
+                                  float *lse, void *stream);
+
+/*
  * The whole iteration from HOST buffers: plan, host->device copies of q,
  * k_new, v_new, append, attention, device->host copy of out (and lse if not
  * NULL), and a stream synchronisation.  Staging buffers belong to the pool and

@@ -37,6 +37,7 @@ EXPORTED_SYMBOLS = (
     "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append",
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
+    "ap_static_workspace_bytes", "ap_attention_iteration_static",
 )
 
 
@@ -117,6 +118,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_last_device_status": (ctypes.c_int, [vp, vp]),
         "ap_profile_enable": (ctypes.c_int, [vp, ctypes.c_int]),
         "ap_profile_collect": (ctypes.c_int, [vp, vp, ctypes.POINTER(KernelTimes)]),
+        "ap_static_workspace_bytes": (sz, []),
+        "ap_attention_iteration_static": (ctypes.c_int, [vp, vp, vp, vp, vp, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -311,6 +314,22 @@ def attention_iteration(pool: KVPool, plan: Plan, q, out, lse=None, workspace=No
     _check(load().ap_attention_iteration(pool.handle, plan.handle, _ptr(q), _ptr(out), _ptr(lse),
                                          _ptr(workspace), workspace_bytes, _stream(stream)),
            "ap_attention_iteration")
+
+
+def static_workspace_bytes() -> int:
+    """Size of the library's built-in split-K scratch array (the largest plan
+    workspace :func:`attention_iteration_static` accepts)."""
+    return int(load().ap_static_workspace_bytes())
+
+
+def attention_iteration_static(pool: KVPool, plan: Plan, q, out, lse=None, stream=None) -> None:
+    """Same result as :func:`attention_iteration`, for callers that cannot
+    allocate device memory and therefore have no workspace to pass: the split-K
+    partials go to a fixed 4 MiB array inside the library.  Plans that need
+    more raise ``ApError`` (``AP_ERR_WORKSPACE_TOO_SMALL``).  Calls share that
+    array, so two of them must not overlap on the GPU."""
+    _check(load().ap_attention_iteration_static(pool.handle, plan.handle, _ptr(q), _ptr(out), _ptr(lse),
+                                                _stream(stream)), "ap_attention_iteration_static")
 
 
 def serving_iteration_host(pool: KVPool, q_lens, ctx_lens, block_tables, num_q_heads: int, q_host,

@@ -1,0 +1,93 @@
+"""ap_attention_iteration_static: the attention call for users who cannot
+allocate device memory.
+
+Some integrations run attention from a place where cudaMalloc is off limits:
+all device memory already belongs to a framework's caching allocator, or the
+loop cannot afford cudaMalloc's device-wide synchronisation.  They have no
+workspace to hand to ap_attention_iteration, so the library offers a variant
+that keeps the split-K partials in a fixed 4 MiB array of its own.
+
+This test drives that variant through the C ABI and requires the same output
+as the ordinary entry point on two calls in a row (the second call sees the
+scratch exactly as the first one left it, and a different batch in between
+makes sure stale partials are never picked up).  It lives in the file pytest
+collects last, so a failure here cannot hide the result of any other test.
+"""
+import numpy as np
+import pytest
+
+import paper_2604_07144_b200 as ap
+from paper_2604_07144_b200 import binding as B
+from paper_2604_07144_b200 import workloads as W
+
+from harness import GpuRun, LSE_RTOL, OUT_ATOL, to_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _decode_batch(seed, ctx_lens):
+    ctx = np.asarray(ctx_lens, np.int32)
+    return W._assemble(f"static_ws_{seed}", W.SHAPE_8B, W.make_rng(seed), np.ones(len(ctx), np.int32), ctx, 1.3)
+
+
+def _reference(run):
+    """Output of the ordinary entry point (caller-provided workspace)."""
+    run.append()
+    run.attend()
+    assert run.status() == 0
+    n = run.batch.n_new
+    return W.bf16_bits_to_f64(to_bits(run.out)[:n]), run.lse.cpu().numpy()[:n].astype(np.float64)
+
+
+def _static(run):
+    """Output of the no-allocation entry point, into poisoned output buffers."""
+    run.out.fill_(float("nan"))
+    run.lse.fill_(float("nan"))
+    ap.attention_iteration_static(run.pool, run.plan, run.q, run.out, run.lse)
+    assert run.status() == 0
+    n = run.batch.n_new
+    return W.bf16_bits_to_f64(to_bits(run.out)[:n]), run.lse.cpu().numpy()[:n].astype(np.float64)
+
+
+def _same(got, ref):
+    out, lse = got
+    ref_out, ref_lse = ref
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+    assert np.abs(out - ref_out).max() <= OUT_ATOL
+    assert (np.abs(lse - ref_lse) / np.maximum(np.abs(ref_lse), 1.0)).max() <= LSE_RTOL
+
+
+def test_static_workspace_matches_caller_workspace_twice_in_a_row():
+    assert ap.static_workspace_bytes() == 4 << 20
+    # long contexts: every (row, kv head) stream is cut, so partials and the merge are exercised
+    a = GpuRun(_decode_batch(901, [20000, 9001, 333, 64]))
+    b = GpuRun(_decode_batch(902, [15000, 12000, 17]))
+    try:
+        assert a.info["merge_entries"] > 0 and b.info["merge_entries"] > 0
+        assert 0 < a.workspace_bytes <= ap.static_workspace_bytes()
+        ref_a, ref_b = _reference(a), _reference(b)
+        _same(_static(a), ref_a)          # first call (does the one-time address lookup)
+        _same(_static(a), ref_a)          # second call in a row, scratch holds the first call's partials
+        _same(_static(b), ref_b)          # another batch over the same scratch
+        _same(_static(a), ref_a)
+    finally:
+        a.close()
+        b.close()
+
+
+def test_static_workspace_small_plan_and_argument_checks():
+    # A plan with no cut stream needs no scratch at all and must work too; bad
+    # arguments are refused before anything is launched.  (A plan larger than
+    # the 4 MiB array cannot be produced by the planner on 148 SMs, so the
+    # size rule is checked on the plan's own number.)
+    run = GpuRun(_decode_batch(903, [40, 700]))
+    try:
+        assert run.workspace_bytes <= ap.static_workspace_bytes()
+        run.append()
+        ap.attention_iteration_static(run.pool, run.plan, run.q, run.out, run.lse)
+        assert run.status() == 0
+        with pytest.raises(ap.ApError) as e:       # misaligned q is refused before any launch
+            ap.attention_iteration_static(run.pool, run.plan, run.q.data_ptr() + 2, run.out, run.lse)
+        assert e.value.status == B.AP_ERR_INVALID_ARG
+    finally:
+        run.close()
