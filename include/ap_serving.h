@@ -167,7 +167,7 @@ int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
  * section:
  *   append_dst    [n_new]             page*16 + slot of every new token row
  *   bt_flat       [n_bt]              used block-table entries, sequences with q_len > 0 concatenated
- *   decode_items  [decode_items][8]   q_row, kv_head, bt_offset, page_begin, page_count, kv_len, part_slot, 0
+ *   decode_items  [decode_items][8]   q_row, kv_head, bt_offset, page_begin, page_count, kv_len, part_slot, merge_index
  *   cta_begin     [n_cta_begin]       item range of decode CTA c is [cta_begin[c], cta_begin[c+1])
  *   merge_entries [merge_entries][4]  q_row, kv_head, part_begin, part_count
  *   prefill_tiles [prefill_tiles][8]  q_row0, rows, q_head, kv_head, bt_offset, pos0, ctx_len, 0
@@ -192,8 +192,10 @@ int ap_kv_append(ap_kv_pool *pool, const ap_plan *plan, const void *k_new, const
 
 /*
  * Attention for every new token of the batch (decode rows: split-K
- * flash-decoding + LSE merge; prefill chunks: causal tiled attention on
- * tcgen05 tensor cores).  The pool must already hold the iteration's tokens.
+ * flash-decoding, the LSE merge done by the last-arriving split; prefill
+ * chunks: causal tiled attention on tcgen05 tensor cores).  The pool must
+ * already hold the iteration's tokens.  Attention calls on the same pool must
+ * not overlap on the GPU (they share the pool's merge arrival counters).
  * q, out: device, 16-byte aligned; lse: device or NULL; workspace: device,
  * 256-byte aligned, at least ap_plan_workspace_bytes() (else
  * WORKSPACE_TOO_SMALL), contents undefined before and after.
@@ -266,7 +268,8 @@ const char *ap_status_string(int status);
  * library launches for this pool is bracketed by CUDA events recorded on the
  * launching stream.  ap_profile_collect synchronises `stream`, adds up the
  * elapsed times per kernel since the last enable/collect, and clears the
- * records.  Index: 0 kv_append, 1 decode split-K, 2 LSE merge, 3 prefill.
+ * records.  Index: 0 kv_append, 1 decode split-K (which also performs the LSE
+ * merge), 2 unused, 3 prefill.
  */
 enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_MERGE = 2, AP_KERNEL_PREFILL = 3, AP_KERNEL_COUNT = 4 };
 typedef struct ap_kernel_times {

@@ -175,8 +175,8 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
                 break;
             }
         }
-        if (cudaMalloc((void **)&p->d_status, sizeof(int)) != cudaSuccess ||
-            cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) {
+        if (cudaMalloc((void **)&p->d_status, sizeof(int) * (1 + kMaxMergeEntries)) != cudaSuccess ||
+            cudaMemset(p->d_status, 0, sizeof(int) * (1 + kMaxMergeEntries)) != cudaSuccess) {
             rc = AP_ERR_CUDA;
             break;
         }
@@ -365,6 +365,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
                         it.page_count = take;
                         it.kv_len = cl;
                         it.part_slot = -1;
+                        it.merge_index = -1;
                         items.push_back(it);
                         cap -= take + kItemCost;
                         pb += take;
@@ -374,7 +375,10 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
                     if (items.size() - first > 1) {
                         MergeEntry m{row0[(size_t)s], g, n_slots, (int32_t)(items.size() - first)};
                         merges.push_back(m);
-                        for (size_t i = first; i < items.size(); ++i) items[i].part_slot = n_slots++;
+                        for (size_t i = first; i < items.size(); ++i) {
+                            items[i].part_slot = n_slots++;
+                            items[i].merge_index = (int32_t)merges.size() - 1;
+                        }
                     }
                 }
             }
@@ -384,6 +388,19 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
         }
     }
     const int n_ctas = cta_begin.empty() ? 0 : (int)cta_begin.size() - 1;
+    // Inside a CTA, items of cut streams go first: their partials are then merged
+    // in mid-kernel, behind the running pipeline, and not in the kernel's tail.
+    for (int c = 0; c < n_ctas; ++c)
+        std::stable_partition(items.begin() + cta_begin[(size_t)c], items.begin() + cta_begin[(size_t)c + 1],
+                              [](const DecodeItem &it) { return it.part_slot >= 0; });
+    // streams are cut at CTA boundaries only, so a CTA has at most two partial items
+    // (the decode kernel relies on it)
+    for (int c = 0; c < n_ctas; ++c) {
+        int partial = 0;
+        for (int32_t i = cta_begin[(size_t)c]; i < cta_begin[(size_t)c + 1]; ++i) partial += items[(size_t)i].part_slot >= 0;
+        if (partial > 2) return AP_ERR_UNSUPPORTED;
+    }
+    if ((int)merges.size() > kMaxMergeEntries) return AP_ERR_UNSUPPORTED;
 
     // ---- prefill tiles, longest first
     std::vector<PrefillTile> tiles;
@@ -489,7 +506,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     info.merge_entries = (int64_t)merges.size();
     info.prefill_tiles = (int64_t)tiles.size();
     info.launches_append = n_new > 0 ? 1 : 0;
-    info.launches_attention = (items.empty() ? 0 : 1) + (merges.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
+    info.launches_attention = (items.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
     *out = plan;
     return AP_OK;
 }
@@ -556,10 +573,6 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
         TimedScope timed(pool, AP_KERNEL_DECODE, st);
         e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
     }
-    if (e == cudaSuccess && plan->info.merge_entries > 0) {
-        TimedScope timed(pool, AP_KERNEL_MERGE, st);
-        e = launch_lse_merge(pool, plan, o_part, lse_part, out, lse, st);
-    }
     if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
         TimedScope timed(pool, AP_KERNEL_PREFILL, st);
         e = launch_prefill(pool, plan, q, out, lse, st);
@@ -584,7 +597,8 @@ int ap_last_device_status(ap_kv_pool *pool, void *stream) {
         return AP_ERR_CUDA;
     }
     if (status != 0) {
-        if (cudaMemsetAsync(pool->d_status, 0, sizeof(int), st) != cudaSuccess ||
+        // a kernel that gave up may have left merge arrival counters behind: clear them too
+        if (cudaMemsetAsync(pool->d_status, 0, sizeof(int) * (1 + kMaxMergeEntries), st) != cudaSuccess ||
             cudaStreamSynchronize(st) != cudaSuccess) {
             (void)cudaGetLastError();
             return AP_ERR_CUDA;

@@ -13,7 +13,10 @@
 // so every MMA row is a real token and no accumulator register is padding.
 // At the end of an item the four warps' (m, l, O) are combined through shared
 // memory and written either as the final bf16 output (item covers the whole
-// context) or as an fp32 partial (o normalised, lse) for the merge kernel.
+// context) or as an fp32 partial (o normalised, lse).  A sixth warp counts the
+// CTA's partials in on a device-wide arrival counter per cut stream; the last
+// one to arrive merges the stream's partials by log-sum-exp and writes the final
+// output while producer and consumers carry on, so no second kernel is needed.
 #include <cuda_bf16.h>
 
 #include "internal.h"
@@ -26,8 +29,11 @@ namespace {
 using namespace ptx;
 
 constexpr int kConsumerWarps = 4;
-constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kDecodeThreads = (kConsumerWarps + 2) * 32;   // consumers, producer, merge warp
 constexpr int kPPS = kDecodePagesPerStage;
+// A stream is only ever cut at a CTA boundary, so a CTA holds at most two items
+// that produce partials (the planner puts them first in the CTA's list).
+constexpr int kMaxPartialItems = 2;
 static_assert(kPPS == kConsumerWarps, "one page of a stage per consumer warp");
 
 template <int D>
@@ -40,7 +46,7 @@ struct DecodeCfg {
     static constexpr int kORow = D + 4;                             // padded fp32 row of the merge buffer
     static constexpr int kMergeWarpFloats = 8 * kORow + 16;         // O[8][D+4], m[8], l[8]
     static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4;
-    static constexpr int kBarrierBytes = 2 * kStages * 8 + 16;
+    static constexpr int kBarrierBytes = (2 * kStages + kMaxPartialItems) * 8 + 16;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kMergeBytes + kBarrierBytes;
     static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte swizzle alignment");
 };
@@ -82,9 +88,9 @@ __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                      const __nv_bfloat16 *__restrict__ q, const DecodeItem *__restrict__ items,
                      const int32_t *__restrict__ cta_begin, const int32_t *__restrict__ bt_flat,
-                     float *__restrict__ o_part, float *__restrict__ lse_part, __nv_bfloat16 *__restrict__ out,
-                     float *__restrict__ lse_out, int Hq, int Hkv, int G, int num_pages, float scale_log2,
-                     int *status) {
+                     const MergeEntry *__restrict__ merges, float *o_part, float *lse_part,
+                     __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out, int Hq, int Hkv, int G,
+                     int num_pages, float scale_log2, int *status) {
     using Cfg = DecodeCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -92,7 +98,9 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
     float *merge = (float *)(smem + Cfg::kStages * Cfg::kStageBytes);
     uint64_t *full = (uint64_t *)((uint8_t *)merge + Cfg::kMergeBytes);
     uint64_t *empty = full + Cfg::kStages;
-    volatile int *abort_flag = (volatile int *)(empty + Cfg::kStages);
+    uint64_t *part_done = empty + Cfg::kStages;      // [kMaxPartialItems], each completes once
+    volatile int *abort_flag = (volatile int *)(part_done + kMaxPartialItems);
+    int *merge_counters = status + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int item_begin = cta_begin[blockIdx.x], item_end = cta_begin[blockIdx.x + 1];
@@ -102,6 +110,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
+        for (int i = 0; i < kMaxPartialItems; ++i) mbar_init(&part_done[i], 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -154,6 +163,82 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                     if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
                 }
                 cur = nxt;
+            }
+        }
+        return;
+    }
+
+    if (warp == kConsumerWarps + 1) {
+        // ---- LSE merge warp, off the critical path.  For each of this CTA's partial items, once the
+        // consumers have written it: count it in on the stream's device-wide arrival counter; the
+        // item that completes the count merges all partials of the stream,
+        //   lse = m* + ln sum_k exp(lse_k - m*),  o = sum_k exp(lse_k - lse) o_k,  m* = max_k lse_k,
+        // and writes the bf16 result.  mbarrier arrive/wait carry the consumers' stores to this
+        // warp (release/acquire at CTA scope); the acq_rel atomic publishes them device-wide and
+        // acquires the other items' partials.
+        for (int pi = 0; pi < kMaxPartialItems && item_begin + pi < item_end; ++pi) {
+            const DecodeItem item = items[item_begin + pi];
+            if (item.part_slot < 0) break;
+            const MergeEntry me = merges[item.merge_index];
+            if (!wait_or_abort(&part_done[pi], 0, abort_flag)) {
+                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                *abort_flag = 1;
+                return;
+            }
+            int last = 0;
+            if (lane == 0) {
+                int old;
+                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                             : "=r"(old) : "l"(merge_counters + item.merge_index) : "memory");
+                last = old == me.part_count - 1;
+                if (last) merge_counters[item.merge_index] = 0;      // ready for the next launch
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (!last) continue;
+            // Pass 1: lse of the whole stream per head (lanes split the partials).  Pass 2: every
+            // lane owns 4 columns and accumulates sum_k exp(lse_k - lse) o_k for all heads; the
+            // loads of a pass do not depend on each other, so they overlap in flight.
+            float lse_tot[8];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+                float mx = -INFINITY;
+                if (h < G)
+                    for (int k = lane; k < me.part_count; k += 32)
+                        mx = fmaxf(mx, __ldcg(lse_part + (size_t)(me.part_begin + k) * G + h));
+#pragma unroll
+                for (int sh = 16; sh >= 1; sh >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, sh));
+                float sm = 0.f;
+                if (h < G)
+                    for (int k = lane; k < me.part_count; k += 32)
+                        sm += __expf(__ldcg(lse_part + (size_t)(me.part_begin + k) * G + h) - mx);
+#pragma unroll
+                for (int sh = 16; sh >= 1; sh >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, sh);
+                lse_tot[h] = mx + __logf(sm);
+            }
+            float4 acc[8];
+#pragma unroll
+            for (int h = 0; h < 8; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+            const bool col_ok = lane * 4 < D;
+#pragma unroll 2
+            for (int k = 0; k < me.part_count; ++k) {
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    if (h < G && col_ok) {
+                        const size_t prow = (size_t)(me.part_begin + k) * G + h;
+                        const float w = __expf(__ldcg(lse_part + prow) - lse_tot[h]);
+                        const float4 o = __ldcg(reinterpret_cast<const float4 *>(o_part + prow * D) + lane);
+                        acc[h].x += w * o.x; acc[h].y += w * o.y; acc[h].z += w * o.z; acc[h].w += w * o.w;
+                    }
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+                if (h < G && col_ok) {
+                    const size_t orow = (size_t)me.q_row * Hq + (size_t)me.kv_head * G + h;
+                    uint2 v = make_uint2(pack_bf16x2(acc[h].x, acc[h].y), pack_bf16x2(acc[h].z, acc[h].w));
+                    *reinterpret_cast<uint2 *>(out + orow * D + lane * 4) = v;
+                    if (lane == 0 && lse_out) lse_out[orow] = lse_tot[h];
+                }
             }
         }
         return;
@@ -306,6 +391,9 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             }
         }
         named_barrier_sync(1, kConsumerWarps * 32);
+        // the partial is complete: hand it to the merge warp
+        if (item.part_slot >= 0 && threadIdx.x == 0 && it - item_begin < kMaxPartialItems)
+            mbar_arrive(&part_done[it - item_begin]);
     }
 }
 
@@ -324,7 +412,7 @@ cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const v
     const float scale_log2 = plan->scale * 1.4426950408889634f;
     decode_splitk_kernel<D><<<(unsigned)plan->info.decode_ctas, kDecodeThreads, Cfg::kSmemBytes, stream>>>(
         pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
-        o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, plan->group,
+        plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, plan->group,
         pool->desc.num_pages, scale_log2, pool->d_status);
     return cudaGetLastError();
 }

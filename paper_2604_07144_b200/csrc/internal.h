@@ -14,6 +14,7 @@
 namespace ap {
 
 constexpr int kPageSize = 16;
+constexpr int kMaxMergeEntries = 4096;   // arrival counters kept per pool (the planner makes < 2 per CTA)
 
 // ---- device work lists (all int32, uploaded as one blob per plan) ---------
 
@@ -27,7 +28,7 @@ struct DecodeItem {
     int32_t page_count;  // pages in the range (>= 1)
     int32_t kv_len;      // attended length of the row (position + 1)
     int32_t part_slot;   // slot in the partial buffers, or -1: write out/lse directly
-    int32_t pad;
+    int32_t merge_index; // entry in the merge list this partial belongs to, or -1
 };
 static_assert(sizeof(DecodeItem) == 32, "DecodeItem layout");
 
@@ -81,7 +82,7 @@ struct ap_kv_pool {
     ap_pool_desc desc{};
     bool owns_planes = false;
     int sm_count = 0;
-    int *d_status = nullptr;
+    int *d_status = nullptr;          // [0] status word, [1 ..] arrival counters of the merge entries
     CUtensorMap k_map{}, v_map{};
     // allocator
     std::vector<int32_t> free_list;     // pages handed out from the back
@@ -124,8 +125,6 @@ cudaError_t launch_kv_append(const ap_kv_pool *pool, const ap_plan *plan, const 
                              const void *v_new, cudaStream_t stream);
 cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                                  float *lse, float *o_part, float *lse_part, cudaStream_t stream);
-cudaError_t launch_lse_merge(const ap_kv_pool *pool, const ap_plan *plan, const float *o_part,
-                             const float *lse_part, void *out, float *lse, cudaStream_t stream);
 cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                            float *lse, cudaStream_t stream);
 

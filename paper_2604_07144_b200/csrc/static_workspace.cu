@@ -55,14 +55,12 @@ int ap_attention_iteration_static(ap_kv_pool *pool, const ap_plan *plan, const v
     if (rc == AP_OK) {
         cudaStream_t st = (cudaStream_t)stream;
         // Every partial slot is written in full by its decode item before the
-        // merge reads it, so nothing left over from an earlier call is ever
-        // read and nothing needs clearing.
+        // last-arriving item of the stream merges them, so nothing left over
+        // from an earlier call is ever read and nothing needs clearing.
         float *o_part = plan->ws.bytes ? (float *)((char *)ws + plan->ws.o_part_off) : nullptr;
         float *lse_part = plan->ws.bytes ? (float *)((char *)ws + plan->ws.lse_part_off) : nullptr;
         cudaError_t e = cudaSuccess;
         if (plan->info.decode_items > 0) e = ap::launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-        if (e == cudaSuccess && plan->info.merge_entries > 0)
-            e = ap::launch_lse_merge(pool, plan, o_part, lse_part, out, lse, st);
         if (e == cudaSuccess && plan->info.prefill_tiles > 0) e = ap::launch_prefill(pool, plan, q, out, lse, st);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
