@@ -6,14 +6,17 @@
 // each, contiguous in HBM -- into a multi-stage shared-memory ring with TMA
 // (128-byte swizzle, completion on mbarriers) and runs ahead across item
 // boundaries, so the pipeline never drains while consumers finish an item.
-// Four consumer warps each own one page of a stage:
+// Eight consumer warps work as two groups of four that take alternate stages of
+// the ring (two warps per scheduler hide each other's MMA and shuffle latency);
+// within its group's stage a warp owns one page:
 //     S^T = K_page Q^T      (mma.sync m16n8k16: M = 16 tokens, N = 8 heads)
 //     online softmax over tokens (fp32, warp shuffles across the token lanes)
 //     O^T += V_page^T P^T   (M = 16 columns of d per tile, N = 8 heads)
 // so every MMA row is a real token and no accumulator register is padding.
-// At the end of an item the four warps' (m, l, O) are combined through shared
-// memory and written either as the final bf16 output (item covers the whole
-// context) or as an fp32 partial (o normalised, lse).  A sixth warp counts the
+// At the end of an item the four warps drop their (m, l, O) into one of two
+// shared-memory buffers and move on; a combine warp folds them and writes either
+// the final bf16 output (item covers the whole context) or an fp32 partial
+// (o normalised, lse), off the consumers' critical path.  A further warp counts the
 // CTA's partials in on a device-wide arrival counter per cut stream; the last
 // one to arrive merges the stream's partials by log-sum-exp and writes the final
 // output while producer and consumers carry on, so no second kernel is needed.
@@ -28,27 +31,28 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kConsumerWarps = 4;
-constexpr int kDecodeThreads = (kConsumerWarps + 2) * 32;   // consumers, producer, merge warp
+constexpr int kConsumerWarps = 8;           // two groups of four; a group takes every other stage of the ring
+constexpr int kDecodeThreads = (kConsumerWarps + 3) * 32;   // consumers, producer, LSE-merge warp, combine warp
 constexpr int kPPS = kDecodePagesPerStage;
 // A stream is only ever cut at a CTA boundary, so a CTA holds at most two items
 // that produce partials (the planner puts them first in the CTA's list).
 constexpr int kMaxPartialItems = 2;
-static_assert(kPPS == kConsumerWarps, "one page of a stage per consumer warp");
+constexpr int kSmemItems = 64;           // item descriptors of a CTA kept in shared memory
+static_assert(2 * kPPS == kConsumerWarps, "one page of a stage per warp of a consumer group");
 
 template <int D>
 struct DecodeCfg {
-    static constexpr int kHalves = D / 64;
     static constexpr int kTileBytes = kPageSize * D * 2;            // one (page, head) tile of one plane
     static constexpr int kQBytes = 8 * D * 2;                       // up to 8 query heads
     static constexpr int kStageBytes = 2 * kPPS * kTileBytes + kQBytes;
-    static constexpr int kStages = D == 128 ? 5 : 8;
+    static constexpr int kStages = D == 128 ? 4 : 8;
     static constexpr int kORow = D + 4;                             // padded fp32 row of the merge buffer
     static constexpr int kMergeWarpFloats = 8 * kORow + 16;         // O[8][D+4], m[8], l[8]
-    static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4;
-    static constexpr int kBarrierBytes = (2 * kStages + kMaxPartialItems) * 8 + 16;
+    static constexpr int kMergeBytes = 2 * kConsumerWarps * kMergeWarpFloats * 4;   // two buffers
+    static constexpr int kBarrierBytes = (2 * kStages + kMaxPartialItems + 4) * 8 + 16 + kSmemItems * 32;
     static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kMergeBytes + kBarrierBytes;
     static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte swizzle alignment");
+    static_assert(kStages % 2 == 0, "consumer groups own alternate ring slots");
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -99,7 +103,10 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
     uint64_t *full = (uint64_t *)((uint8_t *)merge + Cfg::kMergeBytes);
     uint64_t *empty = full + Cfg::kStages;
     uint64_t *part_done = empty + Cfg::kStages;      // [kMaxPartialItems], each completes once
-    volatile int *abort_flag = (volatile int *)(part_done + kMaxPartialItems);
+    uint64_t *item_done = part_done + kMaxPartialItems;   // [2] consumers -> combine warp, per merge buffer
+    uint64_t *buf_free = item_done + 2;                    // [2] combine warp -> consumers
+    volatile int *abort_flag = (volatile int *)(buf_free + 2);
+    DecodeItem *s_items = (DecodeItem *)(buf_free + 4);
     int *merge_counters = status + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -111,10 +118,22 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             mbar_init(&empty[s], kConsumerWarps);
         }
         for (int i = 0; i < kMaxPartialItems; ++i) mbar_init(&part_done[i], 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&item_done[i], kConsumerWarps);
+            mbar_init(&buf_free[i], 1);
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
+    // The CTA's item descriptors go to shared memory once, so that neither the producer nor the
+    // consumers pay a global-memory round trip at every item boundary.
+    {
+        const int n_ints = min(item_end - item_begin, kSmemItems) * (int)(sizeof(DecodeItem) / 4);
+        const int32_t *src = reinterpret_cast<const int32_t *>(items + item_begin);
+        for (int i = threadIdx.x; i < n_ints; i += kDecodeThreads) reinterpret_cast<int32_t *>(s_items)[i] = __ldg(src + i);
+    }
     __syncthreads();
+    auto get_item = [&](int it) -> DecodeItem { return it - item_begin < kSmemItems ? s_items[it - item_begin] : items[it]; };
 
     int stage = 0;
     uint32_t phase = 0;
@@ -125,11 +144,19 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             prefetch_tensormap(&k_map);
             prefetch_tensormap(&v_map);
         }
+        DecodeItem item = get_item(item_begin);
+        int32_t cur = lane < item.page_count ? __ldg(bt_flat + item.bt_offset + item.page_begin + lane) : 0;
         for (int it = item_begin; it < item_end; ++it) {
-            const DecodeItem item = items[it];
             const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
             const int npages = item.page_count;
-            int32_t cur = lane < npages ? __ldg(bt + lane) : 0;
+            // block-table entries of the next item's first pages are fetched one item ahead
+            DecodeItem next_item = item;
+            int32_t next_cur = 0;
+            if (it + 1 < item_end) {
+                next_item = get_item(it + 1);
+                next_cur = lane < next_item.page_count
+                               ? __ldg(bt_flat + next_item.bt_offset + next_item.page_begin + lane) : 0;
+            }
             for (int p0 = 0; p0 < npages; p0 += 32) {
                 const int32_t nxt = p0 + 32 + lane < npages ? __ldg(bt + p0 + 32 + lane) : 0;
                 const int ngroup = min(32, npages - p0);
@@ -141,7 +168,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                         return;
                     }
                     int32_t page = __shfl_sync(0xffffffffu, cur, s0 + (lane & (kPPS - 1)));
-                    const bool first = (p0 == 0 && s0 == 0);
+                    const bool first = p0 == 0 && s0 < 2 * kPPS;   // each consumer group reads Q from its first stage
                     uint8_t *st = stages + stage * Cfg::kStageBytes;
                     if (lane == 0)
                         mbar_arrive_expect_tx(&full[stage], (uint32_t)(n * 2 * Cfg::kTileBytes +
@@ -164,6 +191,8 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                 }
                 cur = nxt;
             }
+            item = next_item;
+            cur = next_cur;
         }
         return;
     }
@@ -177,7 +206,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         // warp (release/acquire at CTA scope); the acq_rel atomic publishes them device-wide and
         // acquires the other items' partials.
         for (int pi = 0; pi < kMaxPartialItems && item_begin + pi < item_end; ++pi) {
-            const DecodeItem item = items[item_begin + pi];
+            const DecodeItem item = get_item(item_begin + pi);
             if (item.part_slot < 0) break;
             const MergeEntry me = merges[item.merge_index];
             if (!wait_or_abort(&part_done[pi], 0, abort_flag)) {
@@ -244,13 +273,73 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         return;
     }
 
+    if (warp == kConsumerWarps + 2) {
+        // ---- combine warp: per item, folds the four consumer warps' (m, l, O) into one result,
+        //   m* = max_w m_w,  L = sum_w 2^((m_w - m*) c) l_w,  o = sum_w 2^((m_w - m*) c) O_w / L,
+        // and writes the final bf16 output (item covers the whole context) or the fp32 partial.
+        const float kLn2 = 0.6931471805599453f;
+        const bool col_ok = lane * 4 < D;
+        for (int it = item_begin; it < item_end; ++it) {
+            const DecodeItem item = get_item(it);
+            const int ti = it - item_begin, buf = ti & 1;
+            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti >> 1) & 1u, abort_flag)) {
+                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                *abort_flag = 1;
+                return;
+            }
+            const float *mb = merge + buf * kConsumerWarps * Cfg::kMergeWarpFloats;
+#pragma unroll
+            for (int h = 0; h < 8; ++h) {
+                if (h >= G) break;
+                float mw[kConsumerWarps], mstar = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    mw[w] = mb[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + h];
+                    mstar = fmaxf(mstar, mw[w]);
+                }
+                float L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float wt = exp2_approx((mw[w] - mstar) * scale_log2);
+                    L += wt * mb[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + 8 + h];
+                    if (col_ok) {
+                        const float4 o = *reinterpret_cast<const float4 *>(mb + w * Cfg::kMergeWarpFloats +
+                                                                            h * Cfg::kORow + lane * 4);
+                        acc.x += wt * o.x; acc.y += wt * o.y; acc.z += wt * o.z; acc.w += wt * o.w;
+                    }
+                }
+                const float inv = 1.f / L;
+                const float lse = (mstar * scale_log2 + log2f(L)) * kLn2;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+                if (item.part_slot < 0) {
+                    const size_t row = (size_t)item.q_row * Hq + (size_t)item.kv_head * G + h;
+                    if (col_ok)
+                        *reinterpret_cast<uint2 *>(out + row * D + lane * 4) =
+                            make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+                    if (lane == 0 && lse_out) lse_out[row] = lse;
+                } else {
+                    const size_t row = (size_t)item.part_slot * G + h;
+                    if (col_ok) *reinterpret_cast<float4 *>(o_part + row * D + lane * 4) = acc;
+                    if (lane == 0) lse_part[row] = lse;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&buf_free[buf]);
+                // the partial is complete: hand it to the merge warp
+                if (item.part_slot >= 0 && ti < kMaxPartialItems) mbar_arrive(&part_done[ti]);
+            }
+        }
+        return;
+    }
+
     // ---------------------------------------------------------- consumers --
     const int g = lane >> 2, t = lane & 3;
-    const float kLn2 = 0.6931471805599453f;
-    float *my_merge = merge + warp * Cfg::kMergeWarpFloats;
+    const int grp = warp / kPPS, slot = warp % kPPS;
 
     for (int it = item_begin; it < item_end; ++it) {
-        const DecodeItem item = items[it];
+        const DecodeItem item = get_item(it);
         const int npages = item.page_count;
         const int valid = min(item.kv_len, (item.page_begin + npages) * kPageSize) - item.page_begin * kPageSize;
 
@@ -259,15 +348,26 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
 #pragma unroll
         for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
         uint32_t qf[D / 16][2];
+        bool have_q = false;
 
         for (int p0 = 0; p0 < npages; p0 += kPPS) {
+            // Every warp passes through every stage, also the other group's: it sees the stage
+            // arrive and signs it off.  A stage is refilled only after all eight warps are past it,
+            // which keeps every waiter within one phase of each barrier (a parity wait is ambiguous
+            // beyond that).
             if (!wait_or_abort(&full[stage], phase, abort_flag)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
+            if ((stage & 1) != grp) {                    // the other group's stage (ring slots alternate)
+                if (lane == 0) mbar_arrive(&empty[stage]);
+                if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+                continue;
+            }
             uint8_t *st = stages + stage * Cfg::kStageBytes;
-            if (p0 == 0) {
+            if (!have_q) {                               // this group's first stage of the item (it carries Q)
+                have_q = true;
                 // Q^T as the B operand: b0 = Q[head g][16ks + 2t, +1], b1 = Q[head g][16ks + 8 + 2t, +1]
                 const uint32_t *qs = (const uint32_t *)(st + 2 * kPPS * Cfg::kTileBytes);
 #pragma unroll
@@ -276,11 +376,11 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                     qf[ks][1] = g < G ? qs[(g * D + ks * 16 + 8 + 2 * t) >> 1] : 0u;
                 }
             }
-            const int my_page = p0 + warp;
+            const int my_page = p0 + slot;
             if (my_page < npages) {
                 const int tv = min(kPageSize, valid - my_page * kPageSize);   // valid tokens in this page (>= 1)
-                const uint32_t k_tile = smem_u32(st + warp * Cfg::kTileBytes);
-                uint8_t *v_ptr = st + (kPPS + warp) * Cfg::kTileBytes;
+                const uint32_t k_tile = smem_u32(st + slot * Cfg::kTileBytes);
+                uint8_t *v_ptr = st + (kPPS + slot) * Cfg::kTileBytes;
                 const uint32_t v_tile = smem_u32(v_ptr);
                 if (tv < kPageSize) {
                     // slots past the context hold no token: clear their V rows so 0 * garbage cannot poison O
@@ -344,7 +444,15 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
         }
 
-        // ---- combine the four warps' (m, l, O)
+        // ---- hand (m, l, O) to the combine warp through one of two shared-memory buffers and go on
+        // with the next item; the buffer is reused two items later, once the combine warp has freed it
+        const int ti = it - item_begin, buf = ti & 1;
+        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti >> 1) & 1u) ^ 1u, abort_flag)) {
+            atomicCAS(status, 0, AP_ERR_TIMEOUT);
+            *abort_flag = 1;
+            return;
+        }
+        float *my_merge = merge + (buf * kConsumerWarps + warp) * Cfg::kMergeWarpFloats;
 #pragma unroll
         for (int sh = 4; sh <= 16; sh <<= 1) {
             l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
@@ -363,37 +471,8 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             my_merge[8 * Cfg::kORow + 8 + 2 * t] = l0;
             my_merge[8 * Cfg::kORow + 8 + 2 * t + 1] = l1;
         }
-        named_barrier_sync(1, kConsumerWarps * 32);
-        for (int idx = threadIdx.x; idx < G * D; idx += kConsumerWarps * 32) {
-            const int head = idx / D, col = idx % D;
-            float mstar = -INFINITY;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w)
-                mstar = fmaxf(mstar, merge[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + head]);
-            float L = 0.f, acc = 0.f;
-#pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
-                const float *mw = merge + w * Cfg::kMergeWarpFloats;
-                const float wt = exp2_approx((mw[8 * Cfg::kORow + head] - mstar) * scale_log2);
-                L += wt * mw[8 * Cfg::kORow + 8 + head];
-                acc += wt * mw[head * Cfg::kORow + col];
-            }
-            const float val = acc / L;
-            const float lse = (mstar * scale_log2 + log2f(L)) * kLn2;
-            if (item.part_slot < 0) {
-                const size_t row = (size_t)item.q_row * Hq + (size_t)item.kv_head * G + head;
-                out[row * D + col] = __float2bfloat16_rn(val);
-                if (col == 0 && lse_out) lse_out[row] = lse;
-            } else {
-                const size_t row = (size_t)item.part_slot * G + head;
-                o_part[row * D + col] = val;
-                if (col == 0) lse_part[row] = lse;
-            }
-        }
-        named_barrier_sync(1, kConsumerWarps * 32);
-        // the partial is complete: hand it to the merge warp
-        if (item.part_slot >= 0 && threadIdx.x == 0 && it - item_begin < kMaxPartialItems)
-            mbar_arrive(&part_done[it - item_begin]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&item_done[buf]);
     }
 }
 
