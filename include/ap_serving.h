@@ -170,7 +170,7 @@ int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
  *   decode_items  [decode_items][8]   q_row, kv_head, bt_offset, page_begin, page_count, kv_len, part_slot, merge_index
  *   cta_begin     [n_cta_begin]       item range of decode CTA c is [cta_begin[c], cta_begin[c+1])
  *   merge_entries [merge_entries][4]  q_row, kv_head, part_begin, part_count
- *   prefill_tiles [prefill_tiles][8]  q_row0, rows, q_head, kv_head, bt_offset, pos0, ctx_len, 0
+ *   prefill_tiles [prefill_tiles][8]  q_row0, rows, q_head, kv_head, bt_offset, pos0, ctx_len, q_head_b (-1: none)
  * blob: host, capacity_ints >= layout.total_ints, or NULL to query the layout only.
  */
 typedef struct ap_plan_layout {

@@ -408,11 +408,13 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
         const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
         if (ql <= 1) continue;
         for (int32_t t0 = 0; t0 < ql; t0 += 128) {
-            for (int h = 0; h < b->num_q_heads; ++h) {
+            // two q heads of one kv head share a work unit (and its K/V stream); an odd head is alone
+            for (int h = 0; h < b->num_q_heads; h += ((h % G) + 1 < G ? 2 : 1)) {
                 PrefillTile t{};
                 t.q_row0 = row0[(size_t)s] + t0;
                 t.rows = std::min(128, ql - t0);
                 t.q_head = h;
+                t.q_head_b = (h % G) + 1 < G ? h + 1 : -1;
                 t.kv_head = h / G;
                 t.bt_offset = bt_off[(size_t)s];
                 t.pos0 = cl - ql + t0;

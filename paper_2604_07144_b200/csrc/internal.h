@@ -50,7 +50,7 @@ struct PrefillTile {
     int32_t bt_offset;
     int32_t pos0;        // position of the first query row in its sequence
     int32_t ctx_len;     // sequence context length (positions >= ctx_len hold no token)
-    int32_t pad;
+    int32_t q_head_b;    // second q head of the same kv head sharing the K/V stream, or -1
 };
 static_assert(sizeof(PrefillTile) == 32, "PrefillTile layout");
 

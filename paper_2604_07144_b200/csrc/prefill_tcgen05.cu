@@ -2,18 +2,26 @@
 // accumulators in tensor memory (TMEM).
 //
 // One CTA handles one work unit: 128 consecutive query rows of one sequence for
-// one q head, over keys 0 .. (position of its last row).  Keys and values come
-// through the block table, one TMA per (page, kv head) tile, straight into the
-// 128-byte-swizzled operand layout tcgen05.mma reads.
+// TWO q heads of the same kv head (tiles A and B; B may be absent), over keys
+// 0 .. (position of the last row).  Both tiles consume the same K/V stream, which
+// comes through the block table, one TMA per (page, kv head) tile, straight into
+// the 128-byte-swizzled operand layout tcgen05.mma reads.
 //
-//   warps 0-3  softmax: thread r owns query row r (= TMEM lane r): reads S from
-//              TMEM, masks, keeps the running max / sum in fp32, writes P (bf16)
-//              to shared memory as the A operand of the second product,
-//              rescales O in TMEM when the running max has moved enough, and
-//              writes the normalised output at the end
-//   warp 4     producer: Q tile once, then K and V tiles into a 2-stage ring
-//   warp 5     MMA issuer: S = Q K^T (8 x M128 N128 K16), O += P V, completion
-//              signalled to the other warps through tcgen05.commit -> mbarrier
+//   warps 0-3   softmax group A: thread r owns query row r of tile A (= TMEM lane r)
+//   warps 4-7   softmax group B: same for tile B
+//               per step of 128 keys: read S from TMEM, mask, running max / sum in
+//               fp32, write P (bf16) back into the S columns of TMEM as the A operand
+//               of the second product, rescale O in TMEM when the running max has
+//               moved enough, and write the normalised output at the end
+//   warp 8      producer: Q tiles once, then K and V tiles into a 2-stage ring
+//   warp 9      MMA issuer: S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
+//               tensor pipe works on one tile while the other tile's softmax runs
+//   warps 10-11 idle (they only complete the third warpgroup for the register split)
+//
+// TMEM columns: S_A/P_A 0-127, S_B/P_B 128-255, O_A 256-.., O_B 384-.. (512 allocated).
+// Registers: the block is launched with 168 registers per thread; the third
+// warpgroup drops to 40 and the two softmax groups raise themselves to 232
+// (128 * 40 + 256 * 232 = 384 * 168), so a whole S row fits in registers.
 //
 // Every wait is bounded; a wait that runs out records AP_ERR_TIMEOUT, raises the
 // CTA's abort flag, and all roles fall through to the common exit where TMEM is
@@ -29,11 +37,12 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kTileM = 128;                 // query rows per CTA
+constexpr int kTileM = 128;                 // query rows per tile
 constexpr int kTileN = 128;                 // keys per step (8 pages)
 constexpr int kPagesPerTile = kTileN / kPageSize;
 constexpr int kKvStages = 2;
-constexpr int kPrefillThreads = 192;
+constexpr int kPrefillThreads = 384;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
 
 template <int D>
@@ -42,16 +51,14 @@ struct PrefillCfg {
     static constexpr int kPageTileBytes = kPageSize * D * 2;
     static constexpr int kQBytes = kTileM * D * 2;
     static constexpr int kKvTileBytes = kTileN * D * 2;
-    static constexpr int kPBytes = kTileM * kTileN * 2;
-    static constexpr int kOffQ = 0;
-    static constexpr int kOffP = kOffQ + kQBytes;
-    static constexpr int kOffK = kOffP + kPBytes;
+    static constexpr int kOffQ = 0;                                   // [2] tiles A, B
+    static constexpr int kOffK = kOffQ + 2 * kQBytes;
     static constexpr int kOffV = kOffK + kKvStages * kKvTileBytes;
     static constexpr int kOffBar = kOffV + kKvStages * kKvTileBytes;
     static constexpr int kSmemBytes = 1024 + kOffBar + 256;
-    static constexpr uint32_t kTmemCols = 256;   // S: 128 columns, O: D columns
-    static constexpr uint32_t kColS = 0;
-    static constexpr uint32_t kColO = 128;
+    static constexpr uint32_t kTmemCols = 512;
+    static constexpr uint32_t kColS = 0;      // + 128 * tile
+    static constexpr uint32_t kColO = 256;    // + 128 * tile
 };
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
@@ -99,16 +106,17 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     uint64_t *bars = (uint64_t *)(smem + Cfg::kOffBar);
     uint64_t *q_full = bars + 0;
     uint64_t *k_full = bars + 1;                 // [kKvStages]
-    uint64_t *v_full = bars + 1 + kKvStages;     // [kKvStages]
-    uint64_t *kv_empty = bars + 1 + 2 * kKvStages;
-    uint64_t *s_full = bars + 1 + 3 * kKvStages;
-    uint64_t *p_full = s_full + 1;
-    uint64_t *pv_done = s_full + 2;
-    uint32_t *tmem_slot = (uint32_t *)(s_full + 3);
+    uint64_t *v_full = k_full + kKvStages;       // [kKvStages]
+    uint64_t *kv_empty = v_full + kKvStages;     // [kKvStages]
+    uint64_t *s_full = kv_empty + kKvStages;     // [2] per tile
+    uint64_t *p_full = s_full + 2;               // [2]
+    uint64_t *o_done = p_full + 2;               // [2]
+    uint32_t *tmem_slot = (uint32_t *)(o_done + 2);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const PrefillTile tile = tiles[blockIdx.x];
+    const int n_tiles = tile.q_head_b >= 0 ? 2 : 1;
     const int kv_len = tile.pos0 + tile.rows;                       // keys the last valid row attends
     const int n_steps = (kv_len + kTileN - 1) / kTileN;
     const int total_pages = (tile.ctx_len + kPageSize - 1) / kPageSize;
@@ -120,13 +128,15 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             mbar_init(&v_full[s], 1);
             mbar_init(&kv_empty[s], 1);
         }
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 128);
-        mbar_init(pv_done, 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&s_full[x], 1);
+            mbar_init(&p_full[x], 128);
+            mbar_init(&o_done[x], 1);
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tmem_alloc(tmem_slot, Cfg::kTmemCols);
         tmem_relinquish();
     }
@@ -135,225 +145,239 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     tcgen05_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
-        // ------------------------------------------------------ producer --
-        if (lane == 0) {
-            prefetch_tensormap(&q_map);
-            prefetch_tensormap(&k_map);
-            prefetch_tensormap(&v_map);
-            mbar_arrive_expect_tx(q_full, Cfg::kQBytes);
-            tma_load_3d(smem + Cfg::kOffQ, &q_map, q_full, 0, tile.q_row0, tile.q_head * Cfg::kHalves);
-        }
-        const int32_t *bt = bt_flat + tile.bt_offset;
-        for (int j = 0; j < n_steps; ++j) {
-            const int s = j % kKvStages;
-            const uint32_t ph = (uint32_t)(j / kKvStages) & 1u;
-            const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
-            int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
-            if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
-                *abort_flag = 1;
-                break;
-            }
+    if (warp >= 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        if (warp == kProducerWarp) {
+            // -------------------------------------------------- producer --
             if (lane == 0) {
-                mbar_arrive_expect_tx(&k_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
-                mbar_arrive_expect_tx(&v_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
+                prefetch_tensormap(&q_map);
+                prefetch_tensormap(&k_map);
+                prefetch_tensormap(&v_map);
+                mbar_arrive_expect_tx(q_full, (uint32_t)(n_tiles * Cfg::kQBytes));
+                tma_load_3d(smem + Cfg::kOffQ, &q_map, q_full, 0, tile.q_row0, tile.q_head * Cfg::kHalves);
+                if (n_tiles == 2)
+                    tma_load_3d(smem + Cfg::kOffQ + Cfg::kQBytes, &q_map, q_full, 0, tile.q_row0,
+                                tile.q_head_b * Cfg::kHalves);
             }
-            __syncwarp();
-            if (lane < np) {
-                if (page < 0 || page >= num_pages) {
-                    atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
-                    page = 0;
-                }
-                const int group = (page * Hkv + tile.kv_head) * 2;
-                tma_load_4d(smem + Cfg::kOffK + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &k_map, &k_full[s],
-                            0, 0, 0, group);
-                tma_load_4d(smem + Cfg::kOffV + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &v_map, &v_full[s],
-                            0, 0, 0, group);
-            }
-        }
-    } else if (warp == 5) {
-        // ---------------------------------------------------- MMA issuer --
-        if (lane == 0) {
-            constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
-            constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
-            const uint32_t q_addr = smem_u32(smem + Cfg::kOffQ);
-            const uint32_t p_addr = smem_u32(smem + Cfg::kOffP);
-            const uint32_t tmem_s = tmem + Cfg::kColS, tmem_o = tmem + Cfg::kColO;
-            bool ok = wait_or_abort(q_full, 0, abort_flag);
-            auto issue_qk = [&](int j) {
+            const int32_t *bt = bt_flat + tile.bt_offset;
+            for (int j = 0; j < n_steps; ++j) {
                 const int s = j % kKvStages;
-                if (!wait_or_abort(&k_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) return false;
-                tcgen05_fence_after();
-                const uint32_t k_addr = smem_u32(smem + Cfg::kOffK + s * Cfg::kKvTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    // Q: [half][128 rows][64], 8-row groups 1024 B apart.  K: [16 groups][half][8][64].
-                    const uint64_t a = smem_desc(q_addr + (ks >> 2) * (kTileM * 128) + (ks & 3) * 32, 16, 1024);
-                    const uint64_t b = smem_desc(k_addr + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 1024 * Cfg::kHalves);
-                    umma_ss(tmem_s, a, b, kIdescQK, ks > 0 ? 1u : 0u);
-                }
-                umma_commit(s_full);
-                return true;
-            };
-            if (ok) ok = issue_qk(0);
-            for (int j = 0; ok && j < n_steps; ++j) {
-                const int s = j % kKvStages;
-                if (!wait_or_abort(p_full, (uint32_t)j & 1u, abort_flag) ||
-                    !wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) {
-                    ok = false;
+                const uint32_t ph = (uint32_t)(j / kKvStages) & 1u;
+                const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
+                int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
+                if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag)) {
+                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    *abort_flag = 1;
                     break;
                 }
-                tcgen05_fence_after();
-                const uint32_t v_addr = smem_u32(smem + Cfg::kOffV + s * Cfg::kKvTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < kTileN / 16; ++ks) {
-                    // P: [half of 64 keys][128 rows][64].  V (MN-major): 16 keys = 2 groups of 8,
-                    // 64-column halves 1024 B apart (LBO), 8-key groups 1024*halves apart (SBO).
-                    const uint64_t a = smem_desc(p_addr + (ks >> 2) * (kTileM * 128) + (ks & 3) * 32, 16, 1024);
-                    const uint64_t b = smem_desc(v_addr + ks * 2 * 1024 * Cfg::kHalves, 1024, 1024 * Cfg::kHalves);
-                    umma_ss(tmem_o, a, b, kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&k_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
+                    mbar_arrive_expect_tx(&v_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
                 }
-                umma_commit(&kv_empty[s]);
-                umma_commit(pv_done);
-                if (j + 1 < n_steps) ok = issue_qk(j + 1);
+                __syncwarp();
+                if (lane < np) {
+                    if (page < 0 || page >= num_pages) {
+                        atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                        page = 0;
+                    }
+                    const int group = (page * Hkv + tile.kv_head) * 2;
+                    tma_load_4d(smem + Cfg::kOffK + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &k_map,
+                                &k_full[s], 0, 0, 0, group);
+                    tma_load_4d(smem + Cfg::kOffV + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &v_map,
+                                &v_full[s], 0, 0, 0, group);
+                }
             }
-            if (!ok) {
+        } else if (warp == kMmaWarp) {
+            // ------------------------------------------------ MMA issuer --
+            if (lane == 0) {
+                constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
+                constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
+                bool ok = wait_or_abort(q_full, 0, abort_flag);
+                // S_x = Q_x K_j^T.  Q: [half][128 rows][64], 8-row groups 1024 B apart.
+                // K: [16 groups of 8 keys][half][8][64].
+                auto issue_qk = [&](int x, int j) {
+                    const int s = j % kKvStages;
+                    const uint32_t q_addr = smem_u32(smem + Cfg::kOffQ + x * Cfg::kQBytes);
+                    const uint32_t k_addr = smem_u32(smem + Cfg::kOffK + s * Cfg::kKvTileBytes);
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint64_t a = smem_desc(q_addr + (ks >> 2) * (kTileM * 128) + (ks & 3) * 32, 16, 1024);
+                        const uint64_t b = smem_desc(k_addr + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 1024 * Cfg::kHalves);
+                        umma_ss(tmem + Cfg::kColS + x * 128, a, b, kIdescQK, ks > 0 ? 1u : 0u);
+                    }
+                    umma_commit(&s_full[x]);
+                };
+                // O_x += P_x V_j.  P: bf16 pairs in the first 64 columns of S_x (A operand from
+                // TMEM, 8 columns per 16 keys).  V (MN-major): 16 keys = 2 groups of 8, 64-column
+                // halves 1024 B apart (LBO), 8-key groups 1024 * halves apart (SBO).
+                auto issue_pv = [&](int x, int j) {
+                    const int s = j % kKvStages;
+                    const uint32_t v_addr = smem_u32(smem + Cfg::kOffV + s * Cfg::kKvTileBytes);
+#pragma unroll
+                    for (int ks = 0; ks < kTileN / 16; ++ks) {
+                        const uint64_t b = smem_desc(v_addr + ks * 2 * 1024 * Cfg::kHalves, 1024, 1024 * Cfg::kHalves);
+                        umma_ts(tmem + Cfg::kColO + x * 128, tmem + Cfg::kColS + x * 128 + ks * 8, b, kIdescPV,
+                                (j > 0 || ks > 0) ? 1u : 0u);
+                    }
+                };
+                if (ok) ok = wait_or_abort(&k_full[0], 0, abort_flag);
+                if (ok) {
+                    tcgen05_fence_after();
+                    for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);
+                }
+                for (int j = 0; ok && j < n_steps; ++j) {
+                    const int s = j % kKvStages;
+                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) { ok = false; break; }
+                    if (j + 1 < n_steps &&
+                        !wait_or_abort(&k_full[(j + 1) % kKvStages], (uint32_t)((j + 1) / kKvStages) & 1u, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    for (int x = 0; x < n_tiles; ++x) {
+                        if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                        tcgen05_fence_after();
+                        issue_pv(x, j);
+                        if (j + 1 < n_steps) issue_qk(x, j + 1);       // overwrites S_x / P_x after the product above
+                        else umma_commit(&o_done[x]);
+                    }
+                    if (!ok) break;
+                    umma_commit(&kv_empty[s]);
+                }
+                if (!ok) {
+                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    *abort_flag = 1;
+                }
+            }
+            __syncwarp();
+        }
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+        // ------------------------------------------------------- softmax --
+        const int x = warp >> 2;                                     // tile A or B
+        if (x < n_tiles) {
+            const int r = threadIdx.x & 127;                         // query row = TMEM lane
+            const int q_head = x == 0 ? tile.q_head : tile.q_head_b;
+            const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+            const uint32_t col_s = Cfg::kColS + x * 128, col_o = Cfg::kColO + x * 128;
+            const int my_pos = min(tile.pos0 + r, tile.ctx_len - 1); // last key this row attends
+            float m_used = -INFINITY, l = 0.f;
+            bool ok = true;
+            for (int j = 0; j < n_steps; ++j) {
+                // S_x(j) complete; the same commit also covers O_x += P_x V of step j-1
+                if (!wait_or_abort(&s_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                uint32_t sreg[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(lane_addr + col_s + c * 32, sreg[c]);
+                tmem_ld_wait();
+                const int tok0 = j * kTileN;
+                float mx = -INFINITY;
+                if (tok0 + kTileN - 1 > tile.pos0) {
+                    // diagonal or last step: keys past the row's position (or past the context) are masked
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            float v = __uint_as_float(sreg[c][i]);
+                            if (tok0 + c * 32 + i > my_pos) v = -INFINITY;
+                            sreg[c][i] = __float_as_uint(v);
+                            mx = fmaxf(mx, v);
+                        }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sreg[c][i]));
+                }
+                // Keep the old reference max unless some row of the warp moved by more than the
+                // threshold: P stays bounded by 2^threshold and O needs no rescale most steps.
+                const float m_new = fmaxf(m_used, mx);
+                const bool moved = (m_new - m_used) * scale_log2 > kRescaleThreshold;   // true while m_used = -inf
+                const bool rescale = __any_sync(0xffffffffu, moved);
+                float alpha = 1.f;
+                if (rescale) {
+                    alpha = exp2_approx((m_used - m_new) * scale_log2);   // 0 on the first step
+                    m_used = m_new;
+                    if (j > 0) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t oreg[32];
+                            tmem_ld_32x32b_x32(lane_addr + col_o + c * 32, oreg);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
+                            tmem_st_32x32b_x32(lane_addr + col_o + c * 32, oreg);
+                        }
+                    }
+                }
+                const float ms = m_used * scale_log2;
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t preg[32];                                  // 64 keys as bf16 pairs
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float p0 = exp2_approx(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i) & 31]) * scale_log2 - ms);
+                        const float p1 = exp2_approx(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i + 1) & 31]) * scale_log2 - ms);
+                        sum += p0 + p1;
+                        preg[i] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st_32x32b_x32(lane_addr + col_s + c * 32, preg);
+                }
+                l = l * alpha + sum;
+                tmem_st_wait();
+                if (x == 0 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
+                    // keys past the context hold no token: clear their V rows so 0 * garbage cannot
+                    // poison O (tile A's group does it; tile B's product is issued after tile A's)
+                    const int s = j % kKvStages;
+                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *v_tile = smem + Cfg::kOffV + s * Cfg::kKvTileBytes;
+                    const int first = tile.ctx_len - tok0;           // first key of the step without a token
+                    for (int idx = r; idx < (kTileN - first) * (D / 8); idx += 128) {
+                        const int key = first + idx / (D / 8), ch = idx % (D / 8);
+                        *(uint4 *)(v_tile + (key >> 3) * (1024 * Cfg::kHalves) + (ch >> 3) * 1024 + (key & 7) * 128 +
+                                   ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();
+                }
+                tcgen05_fence_before();
+                mbar_arrive(&p_full[x]);
+            }
+            if (ok && wait_or_abort(&o_done[x], 0, abort_flag)) {
+                tcgen05_fence_after();
+                const float inv = 1.f / l;
+                const bool valid = r < tile.rows;
+                __nv_bfloat16 *orow = out + ((size_t)(tile.q_row0 + r) * Hq + q_head) * D;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t oreg[32];
+                    tmem_ld_32x32b_x32(lane_addr + col_o + c * 32, oreg);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(oreg[i]) * inv, __uint_as_float(oreg[i + 1]) * inv);
+                            v.y = pack_bf16x2(__uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
+                            v.z = pack_bf16x2(__uint_as_float(oreg[i + 4]) * inv, __uint_as_float(oreg[i + 5]) * inv);
+                            v.w = pack_bf16x2(__uint_as_float(oreg[i + 6]) * inv, __uint_as_float(oreg[i + 7]) * inv);
+                            *(uint4 *)(orow + c * 32 + i) = v;
+                        }
+                    }
+                }
+                if (valid && lse_out)
+                    lse_out[(size_t)(tile.q_row0 + r) * Hq + q_head] =
+                        (m_used * scale_log2 + log2f(l)) * 0.6931471805599453f;
+            } else {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
             }
-        }
-        __syncwarp();
-    } else {
-        // ------------------------------------------------------- softmax --
-        const int r = threadIdx.x;                                   // query row = TMEM lane
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        const int my_pos = min(tile.pos0 + r, tile.ctx_len - 1);     // last key this row attends
-        float m_used = -INFINITY, l = 0.f;
-        uint8_t *p_row = smem + Cfg::kOffP + (r >> 3) * 1024 + (r & 7) * 128;
-        bool ok = true;
-        for (int j = 0; j < n_steps; ++j) {
-            if (!wait_or_abort(s_full, (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
-            tcgen05_fence_after();
-            uint32_t sreg[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(lane_addr + Cfg::kColS + c * 32, sreg[c]);
-            tmem_ld_wait();
-            const int tok0 = j * kTileN;
-            float mx = -INFINITY;
-            if (tok0 + kTileN - 1 > tile.pos0) {
-                // diagonal or last step: keys past the row's position (or past the context) are masked
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float v = __uint_as_float(sreg[c][i]);
-                        if (tok0 + c * 32 + i > my_pos) v = -INFINITY;
-                        sreg[c][i] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
-                    }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sreg[c][i]));
-            }
-            // Keep the old reference max unless some row of the warp moved by more than the
-            // threshold: P stays bounded by 2^threshold and O needs no rescale most steps.
-            const float m_new = fmaxf(m_used, mx);
-            const bool moved = (m_new - m_used) * scale_log2 > kRescaleThreshold;   // true when m_used = -inf
-            const bool rescale = __any_sync(0xffffffffu, moved);
-            float alpha = 1.f;
-            if (rescale) {
-                alpha = exp2_approx((m_used - m_new) * scale_log2);   // 0 on the first step
-                m_used = m_new;
-            }
-            if (j > 0) {
-                // the previous P V product must be done before P is overwritten or O is touched
-                if (!wait_or_abort(pv_done, (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
-                tcgen05_fence_after();
-                if (rescale) {
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t oreg[32];
-                        tmem_ld_32x32b_x32(lane_addr + Cfg::kColO + c * 32, oreg);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
-                        tmem_st_32x32b_x32(lane_addr + Cfg::kColO + c * 32, oreg);
-                    }
-                    tmem_st_wait();
-                }
-            }
-            const float ms = m_used * scale_log2;
-            float sum = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 8) {
-                    float p[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        p[e] = exp2_approx(__uint_as_float(sreg[c][i + e]) * scale_log2 - ms);
-                        sum += p[e];
-                    }
-                    const int chunk = c * 4 + (i >> 3);              // 16-byte chunk = 8 keys
-                    uint4 v = make_uint4(pack_bf16x2(p[0], p[1]), pack_bf16x2(p[2], p[3]), pack_bf16x2(p[4], p[5]),
-                                         pack_bf16x2(p[6], p[7]));
-                    *(uint4 *)(p_row + (chunk >> 3) * (kTileM * 128) + (((chunk & 7) ^ (r & 7)) << 4)) = v;
-                }
-            }
-            l = l * alpha + sum;
-            if (j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
-                // keys past the context hold no token: clear their V rows so 0 * garbage cannot poison O
-                const int s = j % kKvStages;
-                if (!wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) { ok = false; break; }
-                uint8_t *v_tile = smem + Cfg::kOffV + s * Cfg::kKvTileBytes;
-                const int first = tile.ctx_len - tok0;               // first key of the step without a token
-                for (int idx = r; idx < (kTileN - first) * (D / 8); idx += 128) {
-                    const int key = first + idx / (D / 8), ch = idx % (D / 8);
-                    *(uint4 *)(v_tile + (key >> 3) * (1024 * Cfg::kHalves) + (ch >> 3) * 1024 + (key & 7) * 128 +
-                               ((ch & 7) << 4)) = make_uint4(0, 0, 0, 0);
-                }
-            }
-            fence_proxy_async_smem();
-            tcgen05_fence_before();
-            mbar_arrive(p_full);
-        }
-        if (ok && wait_or_abort(pv_done, (uint32_t)(n_steps - 1) & 1u, abort_flag)) {
-            tcgen05_fence_after();
-            const float inv = 1.f / l;
-            const bool valid = r < tile.rows;
-            __nv_bfloat16 *orow = out + ((size_t)(tile.q_row0 + r) * Hq + tile.q_head) * D;
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t oreg[32];
-                tmem_ld_32x32b_x32(lane_addr + Cfg::kColO + c * 32, oreg);
-                tmem_ld_wait();
-                if (valid) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(oreg[i]) * inv, __uint_as_float(oreg[i + 1]) * inv);
-                        v.y = pack_bf16x2(__uint_as_float(oreg[i + 2]) * inv, __uint_as_float(oreg[i + 3]) * inv);
-                        v.z = pack_bf16x2(__uint_as_float(oreg[i + 4]) * inv, __uint_as_float(oreg[i + 5]) * inv);
-                        v.w = pack_bf16x2(__uint_as_float(oreg[i + 6]) * inv, __uint_as_float(oreg[i + 7]) * inv);
-                        *(uint4 *)(orow + c * 32 + i) = v;
-                    }
-                }
-            }
-            if (valid && lse_out)
-                lse_out[(size_t)(tile.q_row0 + r) * Hq + tile.q_head] =
-                    (m_used * scale_log2 + log2f(l)) * 0.6931471805599453f;
-        } else {
-            atomicCAS(status, 0, AP_ERR_TIMEOUT);
-            *abort_flag = 1;
         }
     }
 
     tcgen05_fence_before();
     __syncthreads();
-    if (warp == 5) tmem_dealloc(tmem, Cfg::kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
 template <int D>

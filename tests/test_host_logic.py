@@ -150,11 +150,16 @@ def check_plan_coverage(batch: W.Batch):
         assert it[3] == 0 and it[4] == (int(it[5]) + 15) // 16
     # prefill coverage
     seen_rows = set()
-    for q_row0, nrows, qh, kvh, bt_off, pos0, ctx, _ in ex["prefill_tiles"]:
+    for q_row0, nrows, qh, kvh, bt_off, pos0, ctx, qh_b in ex["prefill_tiles"]:
         assert 1 <= nrows <= 128 and kvh == qh // (hq // hkv)
+        heads = [int(qh)]
+        if qh_b >= 0:                                   # a second head of the same kv head shares the unit
+            assert qh_b == qh + 1 and qh_b // (hq // hkv) == kvh
+            heads.append(int(qh_b))
         for r in range(q_row0, q_row0 + nrows):
-            assert (r, int(qh)) not in seen_rows
-            seen_rows.add((r, int(qh)))
+            for h in heads:
+                assert (r, h) not in seen_rows
+                seen_rows.add((r, h))
         s = int(np.searchsorted(rows, q_row0, side="right") - 1)
         assert ctx == batch.ctx_lens[s] and pos0 == ctx - batch.q_lens[s] + (q_row0 - rows[s])
     want_rows = {(r, h) for s in range(batch.batch) if batch.q_lens[s] > 1
@@ -179,7 +184,7 @@ def test_plan_coverage_full_size_configs():
     i2 = check_plan_coverage(W.config2(with_pool=False))
     assert i2["decode_rows"] == 64 and i2["decode_ctas"] == 148
     i3 = check_plan_coverage(W.config3(with_pool=False))
-    assert i3["prefill_seqs"] == 8 and i3["decode_rows"] == 120 and i3["prefill_tiles"] == 8 * 4 * 32
+    assert i3["prefill_seqs"] == 8 and i3["decode_rows"] == 120 and i3["prefill_tiles"] == 8 * 4 * 16
     i4 = check_plan_coverage(W.config4(with_pool=False))
     assert i4["decode_ctas"] == 148 and i4["merge_entries"] > 0
 
