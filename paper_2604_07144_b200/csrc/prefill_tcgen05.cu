@@ -13,15 +13,15 @@
 //               fp32, write P (bf16) back into the S columns of TMEM as the A operand
 //               of the second product, rescale O in TMEM when the running max has
 //               moved enough, and write the normalised output at the end
-//   warp 8      producer: Q tiles once, then K and V tiles into a 2-stage ring
+//   warp 8      producer: Q tiles once, then K tiles into a 3-stage and V tiles into a 2-stage ring
 //   warp 9      MMA issuer: S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
 //               tensor pipe works on one tile while the other tile's softmax runs
 //   warps 10-11 idle (they only complete the third warpgroup for the register split)
 //
 // TMEM columns: S_A/P_A 0-127, S_B/P_B 128-255, O_A 256-.., O_B 384-.. (512 allocated).
 // Registers: the block is launched with 168 registers per thread; the third
-// warpgroup drops to 40 and the two softmax groups raise themselves to 232
-// (128 * 40 + 256 * 232 = 384 * 168), so a whole S row fits in registers.
+// warpgroup drops to 56 and the two softmax groups raise themselves to 224
+// (128 * 56 + 256 * 224 = 384 * 168), so a whole S row fits in registers.
 //
 // Every wait is bounded; a wait that runs out records AP_ERR_TIMEOUT, raises the
 // CTA's abort flag, and all roles fall through to the common exit where TMEM is
@@ -40,7 +40,8 @@ using namespace ptx;
 constexpr int kTileM = 128;                 // query rows per tile
 constexpr int kTileN = 128;                 // keys per step (8 pages)
 constexpr int kPagesPerTile = kTileN / kPageSize;
-constexpr int kKvStages = 2;
+constexpr int kKStages = 3;                 // K runs further ahead: S(j+1) is issued right after P V of step j
+constexpr int kVStages = 2;
 constexpr int kPrefillThreads = 384;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
@@ -53,8 +54,8 @@ struct PrefillCfg {
     static constexpr int kKvTileBytes = kTileN * D * 2;
     static constexpr int kOffQ = 0;                                   // [2] tiles A, B
     static constexpr int kOffK = kOffQ + 2 * kQBytes;
-    static constexpr int kOffV = kOffK + kKvStages * kKvTileBytes;
-    static constexpr int kOffBar = kOffV + kKvStages * kKvTileBytes;
+    static constexpr int kOffV = kOffK + kKStages * kKvTileBytes;
+    static constexpr int kOffBar = kOffV + kVStages * kKvTileBytes;
     static constexpr int kSmemBytes = 1024 + kOffBar + 256;
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS = 0;      // + 128 * tile
@@ -105,10 +106,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + Cfg::kOffBar);
     uint64_t *q_full = bars + 0;
-    uint64_t *k_full = bars + 1;                 // [kKvStages]
-    uint64_t *v_full = k_full + kKvStages;       // [kKvStages]
-    uint64_t *kv_empty = v_full + kKvStages;     // [kKvStages]
-    uint64_t *s_full = kv_empty + kKvStages;     // [2] per tile
+    uint64_t *k_full = bars + 1;                 // [kKStages]
+    uint64_t *v_full = k_full + kKStages;        // [kVStages]
+    uint64_t *k_empty = v_full + kVStages;       // [kKStages]
+    uint64_t *v_empty = k_empty + kKStages;      // [kVStages]
+    uint64_t *s_full = v_empty + kVStages;       // [2] per tile
     uint64_t *p_full = s_full + 2;               // [2]
     uint64_t *o_done = p_full + 2;               // [2]
     uint32_t *tmem_slot = (uint32_t *)(o_done + 2);
@@ -123,14 +125,17 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < kKvStages; ++s) {
+        for (int s = 0; s < kKStages; ++s) {
             mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        for (int s = 0; s < kVStages; ++s) {
             mbar_init(&v_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+            mbar_init(&v_empty[s], 1);
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&s_full[x], 1);
-            mbar_init(&p_full[x], 128);
+            mbar_init(&p_full[x], 4);            // one arrival per softmax warp
             mbar_init(&o_done[x], 1);
         }
         *abort_flag = 0;
@@ -146,7 +151,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     const uint32_t tmem = *tmem_slot;
 
     if (warp >= 8) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
         if (warp == kProducerWarp) {
             // -------------------------------------------------- producer --
             if (lane == 0) {
@@ -160,31 +165,38 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                                 tile.q_head_b * Cfg::kHalves);
             }
             const int32_t *bt = bt_flat + tile.bt_offset;
-            for (int j = 0; j < n_steps; ++j) {
-                const int s = j % kKvStages;
-                const uint32_t ph = (uint32_t)(j / kKvStages) & 1u;
-                const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
-                int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
-                if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag)) {
-                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
-                    *abort_flag = 1;
-                    break;
-                }
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(&k_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
-                    mbar_arrive_expect_tx(&v_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
-                }
-                __syncwarp();
-                if (lane < np) {
-                    if (page < 0 || page >= num_pages) {
-                        atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
-                        page = 0;
+            // K tiles run one step ahead of V tiles: iteration i loads K_i, then V_(i-1)
+            bool live = true;
+            for (int i = 0; live && i <= n_steps; ++i) {
+#pragma unroll
+                for (int which = 0; which < 2; ++which) {
+                    const int j = which == 0 ? i : i - 1;             // 0: K_j, 1: V_j
+                    if (j < 0 || j >= n_steps) continue;
+                    const int stages = which == 0 ? kKStages : kVStages;
+                    const int s = j % stages;
+                    const uint32_t ph = (uint32_t)(j / stages) & 1u;
+                    uint64_t *full = which == 0 ? &k_full[s] : &v_full[s];
+                    uint64_t *empty = which == 0 ? &k_empty[s] : &v_empty[s];
+                    const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
+                    int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
+                    if (!wait_or_abort(empty, ph ^ 1u, abort_flag)) {
+                        atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                        *abort_flag = 1;
+                        live = false;
+                        break;
                     }
-                    const int group = (page * Hkv + tile.kv_head) * 2;
-                    tma_load_4d(smem + Cfg::kOffK + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &k_map,
-                                &k_full[s], 0, 0, 0, group);
-                    tma_load_4d(smem + Cfg::kOffV + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes, &v_map,
-                                &v_full[s], 0, 0, 0, group);
+                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(np * Cfg::kPageTileBytes));
+                    __syncwarp();
+                    if (lane < np) {
+                        if (page < 0 || page >= num_pages) {
+                            atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                            page = 0;
+                        }
+                        const int group = (page * Hkv + tile.kv_head) * 2;
+                        uint8_t *dst = smem + (which == 0 ? Cfg::kOffK : Cfg::kOffV) + s * Cfg::kKvTileBytes +
+                                       lane * Cfg::kPageTileBytes;
+                        tma_load_4d(dst, which == 0 ? &k_map : &v_map, full, 0, 0, 0, group);
+                    }
                 }
             }
         } else if (warp == kMmaWarp) {
@@ -193,55 +205,63 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
                 constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
                 bool ok = wait_or_abort(q_full, 0, abort_flag);
-                // S_x = Q_x K_j^T.  Q: [half][128 rows][64], 8-row groups 1024 B apart.
-                // K: [16 groups of 8 keys][half][8][64].
+                // Descriptors are built once; per MMA only a constant is added to the address field
+                // (addresses are below 256 KB, so the 14-bit field cannot carry out).
+                // Q: [half][128 rows][64], 8-row groups 1024 B apart.  K: [16 groups of 8 keys][half][8][64].
+                // V (MN-major): 64-column halves 1024 B apart (LBO), 8-key groups 1024 * halves apart (SBO).
+                const uint64_t q_desc0 = smem_desc(smem_u32(smem + Cfg::kOffQ), 16, 1024);
+                const uint64_t k_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 16, 1024 * Cfg::kHalves);
+                const uint64_t v_desc0 = smem_desc(smem_u32(smem + Cfg::kOffV), 1024, 1024 * Cfg::kHalves);
+                // S_x = Q_x K_j^T
                 auto issue_qk = [&](int x, int j) {
-                    const int s = j % kKvStages;
-                    const uint32_t q_addr = smem_u32(smem + Cfg::kOffQ + x * Cfg::kQBytes);
-                    const uint32_t k_addr = smem_u32(smem + Cfg::kOffK + s * Cfg::kKvTileBytes);
+                    const uint64_t a0 = q_desc0 + (uint64_t)((x * Cfg::kQBytes) >> 4);
+                    const uint64_t b0 = k_desc0 + (uint64_t)(((j % kKStages) * Cfg::kKvTileBytes) >> 4);
+                    const uint32_t d = tmem + Cfg::kColS + x * 128;
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint64_t a = smem_desc(q_addr + (ks >> 2) * (kTileM * 128) + (ks & 3) * 32, 16, 1024);
-                        const uint64_t b = smem_desc(k_addr + (ks >> 2) * 1024 + (ks & 3) * 32, 16, 1024 * Cfg::kHalves);
-                        umma_ss(tmem + Cfg::kColS + x * 128, a, b, kIdescQK, ks > 0 ? 1u : 0u);
-                    }
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        umma_ss(d, a0 + (uint64_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4),
+                                b0 + (uint64_t)(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), kIdescQK, ks > 0 ? 1u : 0u);
                     umma_commit(&s_full[x]);
                 };
-                // O_x += P_x V_j.  P: bf16 pairs in the first 64 columns of S_x (A operand from
-                // TMEM, 8 columns per 16 keys).  V (MN-major): 16 keys = 2 groups of 8, 64-column
-                // halves 1024 B apart (LBO), 8-key groups 1024 * halves apart (SBO).
+                // O_x += P_x V_j.  P: bf16 pairs in the first 64 columns of S_x (A operand from TMEM,
+                // 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
                 auto issue_pv = [&](int x, int j) {
-                    const int s = j % kKvStages;
-                    const uint32_t v_addr = smem_u32(smem + Cfg::kOffV + s * Cfg::kKvTileBytes);
+                    const uint64_t b0 = v_desc0 + (uint64_t)(((j % kVStages) * Cfg::kKvTileBytes) >> 4);
+                    const uint32_t d = tmem + Cfg::kColO + x * 128, a = tmem + Cfg::kColS + x * 128;
+                    if (j > 0) {
 #pragma unroll
-                    for (int ks = 0; ks < kTileN / 16; ++ks) {
-                        const uint64_t b = smem_desc(v_addr + ks * 2 * 1024 * Cfg::kHalves, 1024, 1024 * Cfg::kHalves);
-                        umma_ts(tmem + Cfg::kColO + x * 128, tmem + Cfg::kColS + x * 128 + ks * 8, b, kIdescPV,
-                                (j > 0 || ks > 0) ? 1u : 0u);
+                        for (int ks = 0; ks < kTileN / 16; ++ks)
+                            umma_ts(d, a + ks * 8, b0 + (uint64_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), kIdescPV, 1u);
+                    } else {
+#pragma unroll
+                        for (int ks = 0; ks < kTileN / 16; ++ks)
+                            umma_ts(d, a + ks * 8, b0 + (uint64_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), kIdescPV,
+                                    ks > 0 ? 1u : 0u);
                     }
                 };
                 if (ok) ok = wait_or_abort(&k_full[0], 0, abort_flag);
                 if (ok) {
                     tcgen05_fence_after();
                     for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);
+                    umma_commit(&k_empty[0]);
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
-                    const int s = j % kKvStages;
-                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) { ok = false; break; }
-                    if (j + 1 < n_steps &&
-                        !wait_or_abort(&k_full[(j + 1) % kKvStages], (uint32_t)((j + 1) / kKvStages) & 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
+                    if (!wait_or_abort(&v_full[j % kVStages], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
                     for (int x = 0; x < n_tiles; ++x) {
                         if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
                         tcgen05_fence_after();
                         issue_pv(x, j);
-                        if (j + 1 < n_steps) issue_qk(x, j + 1);       // overwrites S_x / P_x after the product above
-                        else umma_commit(&o_done[x]);
+                        if (j + 1 < n_steps) {
+                            if (x == 0 && !wait_or_abort(&k_full[(j + 1) % kKStages], (uint32_t)((j + 1) / kKStages) & 1u,
+                                                         abort_flag)) { ok = false; break; }
+                            issue_qk(x, j + 1);                        // overwrites S_x / P_x after the product above
+                        } else {
+                            umma_commit(&o_done[x]);
+                        }
                     }
                     if (!ok) break;
-                    umma_commit(&kv_empty[s]);
+                    umma_commit(&v_empty[j % kVStages]);
+                    if (j + 1 < n_steps) umma_commit(&k_empty[(j + 1) % kKStages]);
                 }
                 if (!ok) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
@@ -251,7 +271,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             __syncwarp();
         }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
         // ------------------------------------------------------- softmax --
         const int x = warp >> 2;                                     // tile A or B
         if (x < n_tiles) {
@@ -329,8 +349,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 if (x == 0 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
                     // keys past the context hold no token: clear their V rows so 0 * garbage cannot
                     // poison O (tile A's group does it; tile B's product is issued after tile A's)
-                    const int s = j % kKvStages;
-                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kKvStages) & 1u, abort_flag)) { ok = false; break; }
+                    const int s = j % kVStages;
+                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
                     uint8_t *v_tile = smem + Cfg::kOffV + s * Cfg::kKvTileBytes;
                     const int first = tile.ctx_len - tok0;           // first key of the step without a token
                     for (int idx = r; idx < (kTileN - first) * (D / 8); idx += 128) {
@@ -341,7 +361,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     fence_proxy_async_smem();
                 }
                 tcgen05_fence_before();
-                mbar_arrive(&p_full[x]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full[x]);
             }
             if (ok && wait_or_abort(&o_done[x], 0, abort_flag)) {
                 tcgen05_fence_after();
