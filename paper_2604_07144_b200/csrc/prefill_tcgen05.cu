@@ -79,6 +79,32 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
     }
 }
 
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 2^x for two values on the FMA pipe (relieves the special-function unit, which would otherwise
+// bound the softmax): x = n + f with n = round(x), f in [-0.5, 0.5]; 2^f by a cubic fitted for
+// relative error (7.7e-5, well inside the bf16 rounding P gets anyway); 2^n by adding n to the
+// exponent field.  x is clamped at -125 so the exponent cannot wrap (2^-125 is zero for our purposes).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+    const float kMagic = 12582912.f;                       // 1.5 * 2^23: x + kMagic holds round(x) in its low bits
+    x.x = fmaxf(x.x, -125.f);
+    x.y = fmaxf(x.y, -125.f);
+    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 p = __ffma2_rn(f, make_float2(0.05508868f, 0.05508868f), make_float2(0.24260405f, 0.24260405f));
+    p = __ffma2_rn(p, f, make_float2(0.69327624f, 0.69327624f));
+    p = __ffma2_rn(p, f, make_float2(0.99992894f, 0.99992894f));
+    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
+    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
+    return p;
+}
+
 // Shared-memory matrix descriptor for tcgen05.mma, 128-byte swizzle:
 // start address, leading / stride byte offsets (all >> 4), descriptor version 1
 // (bits 46-47), layout type SWIZZLE_128B = 2 (bits 61-63).
@@ -307,7 +333,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sreg[c][i]));
+                        for (int i = 0; i < 32; i += 2)
+                            mx = max3(mx, __uint_as_float(sreg[c][i]), __uint_as_float(sreg[c][i + 1]));
                 }
                 // Keep the old reference max unless some row of the warp moved by more than the
                 // threshold: P stays bounded by 2^threshold and O needs no rescale most steps.
@@ -331,19 +358,30 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     }
                 }
                 const float ms = m_used * scale_log2;
-                float sum = 0.f;
+                const float2 sc2 = make_float2(scale_log2, scale_log2), nms2 = make_float2(-ms, -ms);
+                float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t preg[32];                                  // 64 keys as bf16 pairs
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const float p0 = exp2_approx(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i) & 31]) * scale_log2 - ms);
-                        const float p1 = exp2_approx(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i + 1) & 31]) * scale_log2 - ms);
-                        sum += p0 + p1;
-                        preg[i] = pack_bf16x2(p0, p1);
+                        // two keys at a time on the packed fp32x2 pipe: x = s * c - m * c, then 2^x
+                        float2 xy = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i) & 31]),
+                                                           __uint_as_float(sreg[2 * c + (i >> 4)][(2 * i + 1) & 31])),
+                                               sc2, nms2);
+                        // every other pair goes to the FMA pipe instead of the special-function unit
+                        if (i & 1) {
+                            xy = exp2_poly2(xy);
+                        } else {
+                            xy.x = exp2_approx(xy.x);
+                            xy.y = exp2_approx(xy.y);
+                        }
+                        sum2 = __fadd2_rn(sum2, xy);
+                        preg[i] = pack_bf16x2(xy.x, xy.y);
                     }
                     tmem_st_32x32b_x32(lane_addr + col_s + c * 32, preg);
                 }
+                const float sum = sum2.x + sum2.y;
                 l = l * alpha + sum;
                 tmem_st_wait();
                 if (x == 0 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
