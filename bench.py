@@ -67,7 +67,8 @@ def make_batch(config: int, seed_offset: int = 0, with_pool: bool = True):
     from paper_2604_07144_b200 import workloads as W
     gen = {1: W.config1, 2: W.config2, 3: W.config3, 4: W.config4}[config]
     kw = {} if config == 1 else {"with_pool": with_pool}
-    return gen(seed=W.SEED_BASE + config + 1000 * seed_offset, **kw)
+    from paper_2604_07144_b200 import replicas
+    return gen(seed=replicas.replica_seed(W.SEED_BASE + config, seed_offset), **kw)
 
 
 def algorithmic_bytes(batch, info):
@@ -300,6 +301,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2604_07144_b200 as ap
+    from paper_2604_07144_b200 import replicas
     from paper_2604_07144_b200 import workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
@@ -343,23 +345,14 @@ def main():
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     def reduce_max(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.reduce_max(x, dev)
 
     def reduce_sum(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return replicas.reduce_sum(x, dev)
 
     # ---- device-resident timing
     for i in range(args.warmup):
