@@ -41,7 +41,10 @@ UNIT = "KV-tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitk launch on the
 # bench workload (ncu capture summarised under profiles/), keyed by the hash of
 # the kernel source the counters were taken from; a changed kernel reports null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/decode_splitk_config2.md: 537.0 MB read + 5.1 MB written per launch (algorithmic 535.0 MB)
+    (2, "81d543cbb9225b49"): 542.1e6,
+}
 
 
 def kernel_source_hash() -> str:
