@@ -13,7 +13,7 @@
 //               fp32, write P (bf16) back into the S columns of TMEM as the A operand
 //               of the second product, rescale O in TMEM when the running max has
 //               moved enough, and write the normalised output at the end
-//   warp 8      producer: Q tiles once, then K tiles into a 3-stage and V tiles into a 2-stage ring
+//   warp 8      producer: Q tiles once, then K and V tiles into one 5-slot ring
 //   warp 9      MMA issuer: S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
 //               tensor pipe works on one tile while the other tile's softmax runs
 //   warps 10-11 idle (they only complete the third warpgroup for the register split)
@@ -40,8 +40,13 @@ using namespace ptx;
 constexpr int kTileM = 128;                 // query rows per tile
 constexpr int kTileN = 128;                 // keys per step (8 pages)
 constexpr int kPagesPerTile = kTileN / kPageSize;
-constexpr int kKStages = 3;                 // K runs further ahead: S(j+1) is issued right after P V of step j
-constexpr int kVStages = 2;
+// K and V tiles share one ring of 32 KB slots, filled in the order K_0, K_1, V_0, K_2, V_1, ...
+// (K one step ahead: S(j+1) is issued right after P V of step j).  While one K and one V tile are
+// being consumed, three slots (96 KB) are in flight, which covers the L2 latency at full MMA rate;
+// separate 3 + 2 rings left only one V tile in flight and made the V arrival the period.
+constexpr int kKvSlots = 5;
+__host__ __device__ constexpr int kv_seq_k(int j) { return j == 0 ? 0 : 2 * j - 1; }
+__host__ __device__ inline int kv_seq_v(int j, int n_steps) { return min(2 * j + 2, 2 * n_steps - 1); }
 constexpr int kPrefillThreads = 384;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr float kRescaleThreshold = 8.0f;   // in log2 units: P stays below 2^8
@@ -54,8 +59,7 @@ struct PrefillCfg {
     static constexpr int kKvTileBytes = kTileN * D * 2;
     static constexpr int kOffQ = 0;                                   // [2] tiles A, B
     static constexpr int kOffK = kOffQ + 2 * kQBytes;
-    static constexpr int kOffV = kOffK + kKStages * kKvTileBytes;
-    static constexpr int kOffBar = kOffV + kVStages * kKvTileBytes;
+    static constexpr int kOffBar = kOffK + kKvSlots * kKvTileBytes;
     static constexpr int kSmemBytes = 1024 + kOffBar + 256;
     static constexpr uint32_t kTmemCols = 512;
     static constexpr uint32_t kColS = 0;      // + 128 * tile
@@ -132,11 +136,9 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + Cfg::kOffBar);
     uint64_t *q_full = bars + 0;
-    uint64_t *k_full = bars + 1;                 // [kKStages]
-    uint64_t *v_full = k_full + kKStages;        // [kVStages]
-    uint64_t *k_empty = v_full + kVStages;       // [kKStages]
-    uint64_t *v_empty = k_empty + kKStages;      // [kVStages]
-    uint64_t *s_full = v_empty + kVStages;       // [2] per tile
+    uint64_t *kv_full = bars + 1;                // [kKvSlots]
+    uint64_t *kv_empty = kv_full + kKvSlots;     // [kKvSlots]
+    uint64_t *s_full = kv_empty + kKvSlots;      // [2] per tile
     uint64_t *p_full = s_full + 2;               // [2]
     uint64_t *o_done = p_full + 2;               // [2]
     uint32_t *tmem_slot = (uint32_t *)(o_done + 2);
@@ -151,13 +153,9 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < kKStages; ++s) {
-            mbar_init(&k_full[s], 1);
-            mbar_init(&k_empty[s], 1);
-        }
-        for (int s = 0; s < kVStages; ++s) {
-            mbar_init(&v_full[s], 1);
-            mbar_init(&v_empty[s], 1);
+        for (int s = 0; s < kKvSlots; ++s) {
+            mbar_init(&kv_full[s], 1);
+            mbar_init(&kv_empty[s], 1);
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&s_full[x], 1);
@@ -191,38 +189,31 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                                 tile.q_head_b * Cfg::kHalves);
             }
             const int32_t *bt = bt_flat + tile.bt_offset;
-            // K tiles run one step ahead of V tiles: iteration i loads K_i, then V_(i-1)
-            bool live = true;
-            for (int i = 0; live && i <= n_steps; ++i) {
-#pragma unroll
-                for (int which = 0; which < 2; ++which) {
-                    const int j = which == 0 ? i : i - 1;             // 0: K_j, 1: V_j
-                    if (j < 0 || j >= n_steps) continue;
-                    const int stages = which == 0 ? kKStages : kVStages;
-                    const int s = j % stages;
-                    const uint32_t ph = (uint32_t)(j / stages) & 1u;
-                    uint64_t *full = which == 0 ? &k_full[s] : &v_full[s];
-                    uint64_t *empty = which == 0 ? &k_empty[s] : &v_empty[s];
-                    const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
-                    int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
-                    if (!wait_or_abort(empty, ph ^ 1u, abort_flag)) {
-                        atomicCAS(status, 0, AP_ERR_TIMEOUT);
-                        *abort_flag = 1;
-                        live = false;
-                        break;
+            // ring order K_0, K_1, V_0, K_2, V_1, ...: entry n goes to slot n % kKvSlots
+            const int n_entries = 2 * n_steps;
+            for (int n = 0; n < n_entries; ++n) {
+                // entry n: K_j for n = 0 or odd n < 2 n_steps - 1, else V_j
+                const bool is_k = n == 0 || ((n & 1) && n < n_entries - 1);
+                const int j = is_k ? (n + 1) / 2 : (n == n_entries - 1 ? n_steps - 1 : n / 2 - 1);
+                const int s = n % kKvSlots;
+                const uint32_t ph = (uint32_t)(n / kKvSlots) & 1u;
+                const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
+                int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
+                if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag)) {
+                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    *abort_flag = 1;
+                    break;
+                }
+                if (lane == 0) mbar_arrive_expect_tx(&kv_full[s], (uint32_t)(np * Cfg::kPageTileBytes));
+                __syncwarp();
+                if (lane < np) {
+                    if (page < 0 || page >= num_pages) {
+                        atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                        page = 0;
                     }
-                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)(np * Cfg::kPageTileBytes));
-                    __syncwarp();
-                    if (lane < np) {
-                        if (page < 0 || page >= num_pages) {
-                            atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
-                            page = 0;
-                        }
-                        const int group = (page * Hkv + tile.kv_head) * 2;
-                        uint8_t *dst = smem + (which == 0 ? Cfg::kOffK : Cfg::kOffV) + s * Cfg::kKvTileBytes +
-                                       lane * Cfg::kPageTileBytes;
-                        tma_load_4d(dst, which == 0 ? &k_map : &v_map, full, 0, 0, 0, group);
-                    }
+                    const int group = (page * Hkv + tile.kv_head) * 2;
+                    tma_load_4d(smem + Cfg::kOffK + s * Cfg::kKvTileBytes + lane * Cfg::kPageTileBytes,
+                                is_k ? &k_map : &v_map, &kv_full[s], 0, 0, 0, group);
                 }
             }
         } else if (warp == kMmaWarp) {
@@ -237,11 +228,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 // V (MN-major): 64-column halves 1024 B apart (LBO), 8-key groups 1024 * halves apart (SBO).
                 const uint64_t q_desc0 = smem_desc(smem_u32(smem + Cfg::kOffQ), 16, 1024);
                 const uint64_t k_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 16, 1024 * Cfg::kHalves);
-                const uint64_t v_desc0 = smem_desc(smem_u32(smem + Cfg::kOffV), 1024, 1024 * Cfg::kHalves);
+                const uint64_t v_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 1024, 1024 * Cfg::kHalves);
                 // S_x = Q_x K_j^T
                 auto issue_qk = [&](int x, int j) {
                     const uint64_t a0 = q_desc0 + (uint64_t)((x * Cfg::kQBytes) >> 4);
-                    const uint64_t b0 = k_desc0 + (uint64_t)(((j % kKStages) * Cfg::kKvTileBytes) >> 4);
+                    const uint64_t b0 = k_desc0 + (uint64_t)(((kv_seq_k(j) % kKvSlots) * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColS + x * 128;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
@@ -252,7 +243,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 // O_x += P_x V_j.  P: bf16 pairs in the first 64 columns of S_x (A operand from TMEM,
                 // 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
                 auto issue_pv = [&](int x, int j) {
-                    const uint64_t b0 = v_desc0 + (uint64_t)(((j % kVStages) * Cfg::kKvTileBytes) >> 4);
+                    const uint64_t b0 = v_desc0 + (uint64_t)(((kv_seq_v(j, n_steps) % kKvSlots) * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColO + x * 128, a = tmem + Cfg::kColS + x * 128;
                     if (j > 0) {
 #pragma unroll
@@ -265,20 +256,21 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                                     ks > 0 ? 1u : 0u);
                     }
                 };
-                if (ok) ok = wait_or_abort(&k_full[0], 0, abort_flag);
+                if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag);
                 if (ok) {
                     tcgen05_fence_after();
                     for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);
-                    umma_commit(&k_empty[0]);
+                    umma_commit(&kv_empty[0]);
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
-                    if (!wait_or_abort(&v_full[j % kVStages], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
+                    const int nv = kv_seq_v(j, n_steps), nk = kv_seq_k(j + 1);
+                    if (!wait_or_abort(&kv_full[nv % kKvSlots], (uint32_t)(nv / kKvSlots) & 1u, abort_flag)) { ok = false; break; }
                     for (int x = 0; x < n_tiles; ++x) {
                         if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
                         tcgen05_fence_after();
                         issue_pv(x, j);
                         if (j + 1 < n_steps) {
-                            if (x == 0 && !wait_or_abort(&k_full[(j + 1) % kKStages], (uint32_t)((j + 1) / kKStages) & 1u,
+                            if (x == 0 && !wait_or_abort(&kv_full[nk % kKvSlots], (uint32_t)(nk / kKvSlots) & 1u,
                                                          abort_flag)) { ok = false; break; }
                             issue_qk(x, j + 1);                        // overwrites S_x / P_x after the product above
                         } else {
@@ -286,8 +278,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         }
                     }
                     if (!ok) break;
-                    umma_commit(&v_empty[j % kVStages]);
-                    if (j + 1 < n_steps) umma_commit(&k_empty[(j + 1) % kKStages]);
+                    umma_commit(&kv_empty[nv % kKvSlots]);
+                    if (j + 1 < n_steps) umma_commit(&kv_empty[nk % kKvSlots]);
                 }
                 if (!ok) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
@@ -387,9 +379,9 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 if (x == 0 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
                     // keys past the context hold no token: clear their V rows so 0 * garbage cannot
                     // poison O (tile A's group does it; tile B's product is issued after tile A's)
-                    const int s = j % kVStages;
-                    if (!wait_or_abort(&v_full[s], (uint32_t)(j / kVStages) & 1u, abort_flag)) { ok = false; break; }
-                    uint8_t *v_tile = smem + Cfg::kOffV + s * Cfg::kKvTileBytes;
+                    const int nv = kv_seq_v(j, n_steps), s = nv % kKvSlots;
+                    if (!wait_or_abort(&kv_full[s], (uint32_t)(nv / kKvSlots) & 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *v_tile = smem + Cfg::kOffK + s * Cfg::kKvTileBytes;
                     const int first = tile.ctx_len - tok0;           // first key of the step without a token
                     for (int idx = r; idx < (kTileN - first) * (D / 8); idx += 128) {
                         const int key = first + idx / (D / 8), ch = idx % (D / 8);
