@@ -20,8 +20,8 @@
 //
 // TMEM columns: S_A/P_A 0-127, S_B/P_B 128-255, O_A 256-.., O_B 384-.. (512 allocated).
 // Registers: the block is launched with 168 registers per thread; the third
-// warpgroup drops to 56 and the two softmax groups raise themselves to 224
-// (128 * 56 + 256 * 224 = 384 * 168), so a whole S row fits in registers.
+// warpgroup drops to 72 and the two softmax groups raise themselves to 216
+// (128 * 72 + 256 * 216 = 384 * 168), so a whole S row fits in registers.
 //
 // Every wait is bounded; a wait that runs out records AP_ERR_TIMEOUT, raises the
 // CTA's abort flag, and all roles fall through to the common exit where TMEM is
@@ -175,7 +175,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     const uint32_t tmem = *tmem_slot;
 
     if (warp >= 8) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == kProducerWarp) {
             // -------------------------------------------------- producer --
             if (lane == 0) {
@@ -289,7 +289,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             __syncwarp();
         }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         // ------------------------------------------------------- softmax --
         const int x = warp >> 2;                                     // tile A or B
         if (x < n_tiles) {
