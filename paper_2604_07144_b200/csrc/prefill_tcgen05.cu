@@ -229,37 +229,41 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 const uint64_t q_desc0 = smem_desc(smem_u32(smem + Cfg::kOffQ), 16, 1024);
                 const uint64_t k_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 16, 1024 * Cfg::kHalves);
                 const uint64_t v_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 1024, 1024 * Cfg::kHalves);
-                // S_x = Q_x K_j^T
-                auto issue_qk = [&](int x, int j) {
-                    const uint64_t a0 = q_desc0 + (uint64_t)((x * Cfg::kQBytes) >> 4);
-                    const uint64_t b0 = k_desc0 + (uint64_t)(((kv_seq_k(j) % kKvSlots) * Cfg::kKvTileBytes) >> 4);
+                const uint32_t q_lo = (uint32_t)q_desc0, q_hi = (uint32_t)(q_desc0 >> 32);
+                const uint32_t k_lo = (uint32_t)k_desc0, k_hi = (uint32_t)(k_desc0 >> 32);
+                const uint32_t v_lo = (uint32_t)v_desc0, v_hi = (uint32_t)(v_desc0 >> 32);
+                // S_x = Q_x K^T with K in ring slot `slot`
+                auto issue_qk = [&](int x, int slot) {
+                    const uint32_t a0 = q_lo + (uint32_t)((x * Cfg::kQBytes) >> 4);
+                    const uint32_t b0 = k_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColS + x * 128;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(d, a0 + (uint64_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4),
-                                b0 + (uint64_t)(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), kIdescQK, ks > 0 ? 1u : 0u);
+                        umma_ss_w(d, a0 + (uint32_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4), q_hi,
+                                  b0 + (uint32_t)(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), k_hi, kIdescQK,
+                                  ks > 0 ? 1u : 0u);
                     umma_commit(&s_full[x]);
                 };
-                // O_x += P_x V_j.  P: bf16 pairs in the first 64 columns of S_x (A operand from TMEM,
-                // 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
-                auto issue_pv = [&](int x, int j) {
-                    const uint64_t b0 = v_desc0 + (uint64_t)(((kv_seq_v(j, n_steps) % kKvSlots) * Cfg::kKvTileBytes) >> 4);
+                // O_x += P_x V with V in ring slot `slot`.  P: bf16 pairs in the first 64 columns of S_x
+                // (A operand from TMEM, 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
+                auto issue_pv = [&](int x, int slot, bool first_step) {
+                    const uint32_t b0 = v_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColO + x * 128, a = tmem + Cfg::kColS + x * 128;
-                    if (j > 0) {
+                    if (!first_step) {
 #pragma unroll
                         for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts(d, a + ks * 8, b0 + (uint64_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), kIdescPV, 1u);
+                            umma_ts_w(d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV, 1u);
                     } else {
 #pragma unroll
                         for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts(d, a + ks * 8, b0 + (uint64_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), kIdescPV,
-                                    ks > 0 ? 1u : 0u);
+                            umma_ts_w(d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV,
+                                      ks > 0 ? 1u : 0u);
                     }
                 };
                 if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag);
                 if (ok) {
                     tcgen05_fence_after();
-                    for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);
+                    for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);     // K_0 is ring entry 0, slot 0
                     umma_commit(&kv_empty[0]);
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
@@ -268,11 +272,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     for (int x = 0; x < n_tiles; ++x) {
                         if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
                         tcgen05_fence_after();
-                        issue_pv(x, j);
+                        issue_pv(x, nv % kKvSlots, j == 0);
                         if (j + 1 < n_steps) {
                             if (x == 0 && !wait_or_abort(&kv_full[nk % kKvSlots], (uint32_t)(nk / kKvSlots) & 1u,
                                                          abort_flag)) { ok = false; break; }
-                            issue_qk(x, j + 1);                        // overwrites S_x / P_x after the product above
+                            issue_qk(x, nk % kKvSlots);                // overwrites S_x / P_x after the product above
                         } else {
                             umma_commit(&o_done[x]);
                         }
