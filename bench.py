@@ -139,6 +139,29 @@ class ClockSampler:
         return out
 
 
+def pick_sequences(active, cost, run_seconds, target_s):
+    """Whole sequences of the batch, in batch order, whose estimated oracle time stays within
+    target_s.  The rate comes from a probe on the median-cost sequence and is refined once from a
+    real run if the probe (dominated by fixed overheads) underestimated it."""
+    probe = sorted(active, key=lambda s: cost[s])[len(active) // 2]
+    rate = cost[probe] / max(run_seconds([probe]), 1e-6)
+    chosen = []
+    for _ in range(3):
+        chosen, est = [], 0.0
+        for s in active:
+            if chosen and est + cost[s] / rate > target_s:
+                continue
+            chosen.append(s)
+            est += cost[s] / rate
+        if len(chosen) == len(active):
+            break
+        new_rate = sum(cost[s] for s in chosen) / max(run_seconds(chosen), 1e-6)
+        if new_rate < 1.5 * rate:
+            break
+        rate = new_rate
+    return chosen
+
+
 def cpu_oracle_baseline(batch, target_s: float = 12.0):
     """The oracle as it stands, timed on the host cores on a bounded sample of
     the same workload: whole sequences of the batch, in batch order, until the
@@ -160,15 +183,7 @@ def cpu_oracle_baseline(batch, target_s: float = 12.0):
     active = [int(s) for s in np.nonzero(batch.q_lens > 0)[0]]
     # cost of a sequence ~ q_len * ctx_len
     cost = {s: float(batch.q_lens[s]) * float(batch.ctx_lens[s]) for s in active}
-    probe = min(active, key=lambda s: cost[s])
-    t_probe, _ = run([probe])
-    rate = cost[probe] / max(t_probe, 1e-6)
-    chosen, est = [], 0.0
-    for s in active:
-        if chosen and est + cost[s] / rate > target_s:
-            continue
-        chosen.append(s)
-        est += cost[s] / rate
+    chosen = pick_sequences(active, cost, lambda seqs: run(seqs)[0], target_s)
     t, toks = run(chosen)
     return {"value": toks / t, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"{len(chosen)} of {len(active)} sequences of the workload ({toks} KV-tokens, "
@@ -186,20 +201,18 @@ def run_reference(args):
     k, v = batch.k_pool.copy(), batch.v_pool.copy()
     rows = batch.q_indptr
     active = [int(s) for s in np.nonzero(batch.q_lens > 0)[0]]
-    # bounded sample: the sequences with the smallest q_len*ctx_len cost first, ~2 s per step
-    t0 = time.perf_counter()
+    # bounded sample: whole sequences in batch order, ~2 s of oracle time per step
     oracle.kv_append(k, v, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.k_new, batch.v_new)
-    s0 = min(active, key=lambda s: float(batch.q_lens[s]) * float(batch.ctx_lens[s]))
-    ql = np.zeros_like(batch.q_lens); ql[s0] = batch.q_lens[s0]
-    t1 = time.perf_counter()
-    oracle.attention(k, v, ql, batch.ctx_lens, batch.block_tables, batch.q[rows[s0]:rows[s0 + 1]])
-    rate = float(batch.q_lens[s0]) * float(batch.ctx_lens[s0]) / max(time.perf_counter() - t1, 1e-6)
-    chosen, est = [], 0.0
-    for s in active:
-        c = float(batch.q_lens[s]) * float(batch.ctx_lens[s]) / rate
-        if chosen and est + c > 2.0:
-            continue
-        chosen.append(s); est += c
+    cost = {s: float(batch.q_lens[s]) * float(batch.ctx_lens[s]) for s in active}
+
+    def run_seconds(seqs):
+        ql_ = np.zeros_like(batch.q_lens); ql_[seqs] = batch.q_lens[seqs]
+        q_ = np.concatenate([batch.q[rows[s]:rows[s + 1]] for s in seqs])
+        t1 = time.perf_counter()
+        oracle.attention(k, v, ql_, batch.ctx_lens, batch.block_tables, q_)
+        return time.perf_counter() - t1
+
+    chosen = pick_sequences(active, cost, run_seconds, 2.0)
     ql = np.zeros_like(batch.q_lens); ql[chosen] = batch.q_lens[chosen]
     qsel = np.concatenate([batch.q[rows[s]:rows[s + 1]] for s in chosen])
     knew = np.concatenate([batch.k_new[rows[s]:rows[s + 1]] for s in chosen])
