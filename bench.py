@@ -84,7 +84,22 @@ def algorithmic_bytes(batch, info):
     decode_bytes = decode_kv * per_kv_token + int(dec.sum()) * per_row + int(((batch.ctx_lens[dec] + 15) // 16).sum()) * 4
     append_bytes = 2 * info["n_new"] * 2 * hkv * d * 2     # read + write, K and V
     total = info["kv_tokens"] * per_kv_token + info["n_new"] * per_row + append_bytes
-    return {"per_kv_token": per_kv_token, "decode_kernel": decode_bytes, "total": total}
+    pre = batch.q_lens > 1
+    prefill_rows = int(batch.q_lens[pre].astype(np.int64).sum())
+    prefill_kv = int(batch.ctx_lens[pre].astype(np.int64).sum())
+    prefill_bytes = prefill_kv * per_kv_token + prefill_rows * per_row
+    return {"per_kv_token": per_kv_token, "decode_kernel": decode_bytes, "prefill_kernel": prefill_bytes,
+            "append_kernel": append_bytes, "total": total,
+            "decode_flops": 4 * hq * d * decode_kv, "prefill_flops": 4 * hq * d * info["prefill_pairs"]}
+
+
+def paper_model_us(flops: float, bytes_: float, peaks) -> float:
+    """Operator time by the paper's own cost model (App. B, Eq. "roofline"):
+    pi = min(F/A * B_g, F_g), T_op = F / pi, with the measured copy bandwidth and bf16 peak of this GPU."""
+    if flops <= 0 or bytes_ <= 0:
+        return 0.0
+    pi = min(flops / bytes_ * peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops"] * 1e12)
+    return flops / pi * 1e6
 
 
 class ClockSampler:
@@ -464,6 +479,12 @@ def main():
                 "decode_items", "decode_ctas", "merge_entries", "prefill_tiles")}},
             "roofline": roofline,
             "kernels": kernels,
+            "paper_model_us": {"decode_splitk": paper_model_us(alg["decode_flops"], alg["decode_kernel"], peaks),
+                               "prefill": paper_model_us(alg["prefill_flops"], alg["prefill_kernel"], peaks),
+                               "note": "T_op = F / min(F/A * B, F_peak) with this GPU's measured copy bandwidth and "
+                                       "bf16 peak; compare with kernels.*.us_per_launch"},
+            "prefill_tflops": (alg["prefill_flops"] / (kernels["prefill"]["us_per_launch"] * 1e-6) / 1e12
+                               if kernels.get("prefill", {}).get("us_per_launch") else None),
             "step_gbs": alg["total"] / (ms_per_step * 1e-3) / 1e9,
             "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
         }

@@ -162,3 +162,12 @@ def test_config5_trace_parity():
         print(f"config5 (80 iterations): {checked} sampled outputs, out err {worst[0]:.2e} lse err {worst[1]:.2e}")
     finally:
         run.close()
+
+
+@pytest.mark.parametrize("shape", [(6, 2, 128), (4, 4, 64), (5, 1, 128), (8, 2, 64)],
+                         ids=lambda s: f"Hq{s[0]}_Hkv{s[1]}_d{s[2]}")
+def test_prefill_head_ratios(shape):
+    # odd groups leave a head without a partner (single-tile units); G = 1 has no pairs at all
+    b = W._assemble("prefill_heads", shape, W.make_rng(600), np.array([150, 1, 70], np.int32),
+                    np.array([333, 90, 70], np.int32), 1.3)
+    check_batch_full(b)
