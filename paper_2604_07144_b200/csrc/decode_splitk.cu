@@ -87,6 +87,96 @@ __device__ __forceinline__ uint32_t tile_off(int tok, int chunk) {
                       (((chunk & 7) ^ (tok & 7)) << 4));
 }
 
+// One warp merges the partials of a cut stream,
+//   lse = m* + ln sum_k exp(lse_k - m*),  o = sum_k exp(lse_k - lse) o_k,  m* = max_k lse_k,
+// and writes the bf16 result.  The merge often sits in the kernel's tail, so it is laid out for
+// latency: lane k holds the lse of partial k for all heads (one batch of loads), the weights then
+// travel by shuffle, and the o rows are fetched a batch of up to 16 independent 16-byte loads per lane at
+// a time (lane = 4 columns of d).  Streams of more than 32 partials take the same path in chunks,
+// re-reading the lse values from L2 instead of keeping them in registers.
+template <int D, int G>
+__device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o_part, const float *lse_part,
+                                             __nv_bfloat16 *out, float *lse_out, int Hq, int lane) {
+    const int n = me.part_count;
+    const float *lse_base = lse_part + (size_t)me.part_begin * G;
+    // ---- lse of the whole stream, per head
+    float v[G], mx[G], sm[G], lse_tot[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) mx[h] = -INFINITY;
+    for (int k0 = 0; k0 < n; k0 += 32) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * G + h) : -INFINITY;
+#pragma unroll
+        for (int h = 0; h < G; ++h) mx[h] = fmaxf(mx[h], v[h]);
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], sh));
+        sm[h] = 0.f;
+    }
+    for (int k0 = 0; k0 < n; k0 += 32) {
+        if (n > 32) {
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+                v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * G + h) : -INFINITY;
+        }
+#pragma unroll
+        for (int h = 0; h < G; ++h) sm[h] += __expf(v[h] - mx[h]);
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+#pragma unroll
+        for (int sh = 16; sh >= 1; sh >>= 1) sm[h] += __shfl_xor_sync(0xffffffffu, sm[h], sh);
+        lse_tot[h] = mx[h] + __logf(sm[h]);
+    }
+    // ---- weighted sum of the partial outputs
+    constexpr int kBatch = G <= 4 ? 16 / G : 1;       // partials fetched per batch (up to 16 loads in flight per lane)
+    float4 acc[G];
+#pragma unroll
+    for (int h = 0; h < G; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const bool col_ok = lane * 4 < D;
+    const float4 *o_base = reinterpret_cast<const float4 *>(o_part + (size_t)me.part_begin * G * D) + lane;
+    for (int c0 = 0; c0 < n; c0 += 32) {
+        float w[G];                                    // this lane's partial (c0 + lane): weight per head
+        if (n > 32) {
+#pragma unroll
+            for (int h = 0; h < G; ++h)
+                v[h] = c0 + lane < n ? __ldcg(lse_base + (size_t)(c0 + lane) * G + h) : -INFINITY;
+        }
+#pragma unroll
+        for (int h = 0; h < G; ++h) w[h] = __expf(v[h] - lse_tot[h]);
+        const int cn = min(32, n - c0);
+        for (int k0 = 0; k0 < cn; k0 += kBatch) {
+            float4 o[kBatch][G];
+#pragma unroll
+            for (int kk = 0; kk < kBatch; ++kk)
+#pragma unroll
+                for (int h = 0; h < G; ++h)
+                    o[kk][h] = (k0 + kk < cn && col_ok)
+                                   ? __ldcg(o_base + ((size_t)(c0 + k0 + kk) * G + h) * (D / 4))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int kk = 0; kk < kBatch; ++kk)
+#pragma unroll
+                for (int h = 0; h < G; ++h) {
+                    const float wk = __shfl_sync(0xffffffffu, w[h], (k0 + kk) & 31);
+                    acc[h].x += wk * o[kk][h].x; acc[h].y += wk * o[kk][h].y;
+                    acc[h].z += wk * o[kk][h].z; acc[h].w += wk * o[kk][h].w;
+                }
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        if (col_ok) {
+            const size_t orow = (size_t)me.q_row * Hq + (size_t)me.kv_head * G + h;
+            *reinterpret_cast<uint2 *>(out + orow * D + lane * 4) =
+                make_uint2(pack_bf16x2(acc[h].x, acc[h].y), pack_bf16x2(acc[h].z, acc[h].w));
+            if (lane == 0 && lse_out) lse_out[orow] = lse_tot[h];
+        }
+    }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kDecodeThreads, 1)
 decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
@@ -224,50 +314,15 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             }
             last = __shfl_sync(0xffffffffu, last, 0);
             if (!last) continue;
-            // Pass 1: lse of the whole stream per head (lanes split the partials).  Pass 2: every
-            // lane owns 4 columns and accumulates sum_k exp(lse_k - lse) o_k for all heads; the
-            // loads of a pass do not depend on each other, so they overlap in flight.
-            float lse_tot[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                float mx = -INFINITY;
-                if (h < G)
-                    for (int k = lane; k < me.part_count; k += 32)
-                        mx = fmaxf(mx, __ldcg(lse_part + (size_t)(me.part_begin + k) * G + h));
-#pragma unroll
-                for (int sh = 16; sh >= 1; sh >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, sh));
-                float sm = 0.f;
-                if (h < G)
-                    for (int k = lane; k < me.part_count; k += 32)
-                        sm += __expf(__ldcg(lse_part + (size_t)(me.part_begin + k) * G + h) - mx);
-#pragma unroll
-                for (int sh = 16; sh >= 1; sh >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, sh);
-                lse_tot[h] = mx + __logf(sm);
-            }
-            float4 acc[8];
-#pragma unroll
-            for (int h = 0; h < 8; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const bool col_ok = lane * 4 < D;
-#pragma unroll 2
-            for (int k = 0; k < me.part_count; ++k) {
-#pragma unroll
-                for (int h = 0; h < 8; ++h) {
-                    if (h < G && col_ok) {
-                        const size_t prow = (size_t)(me.part_begin + k) * G + h;
-                        const float w = __expf(__ldcg(lse_part + prow) - lse_tot[h]);
-                        const float4 o = __ldcg(reinterpret_cast<const float4 *>(o_part + prow * D) + lane);
-                        acc[h].x += w * o.x; acc[h].y += w * o.y; acc[h].z += w * o.z; acc[h].w += w * o.w;
-                    }
-                }
-            }
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h < G && col_ok) {
-                    const size_t orow = (size_t)me.q_row * Hq + (size_t)me.kv_head * G + h;
-                    uint2 v = make_uint2(pack_bf16x2(acc[h].x, acc[h].y), pack_bf16x2(acc[h].z, acc[h].w));
-                    *reinterpret_cast<uint2 *>(out + orow * D + lane * 4) = v;
-                    if (lane == 0 && lse_out) lse_out[orow] = lse_tot[h];
-                }
+            switch (G) {
+                case 1: merge_stream<D, 1>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 2: merge_stream<D, 2>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 3: merge_stream<D, 3>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 4: merge_stream<D, 4>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 5: merge_stream<D, 5>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 6: merge_stream<D, 6>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                case 7: merge_stream<D, 7>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+                default: merge_stream<D, 8>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
             }
         }
         return;
