@@ -317,10 +317,29 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
             }
         }
         row0[(size_t)B] = (int32_t)r;
-        // no two appended slots may alias
-        std::vector<int32_t> sorted(append_dst);
-        std::sort(sorted.begin(), sorted.end());
-        if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AP_ERR_BAD_BLOCK_TABLE;
+        // No two appended slots may alias.  A sequence's new tokens fill a slot range in each page
+        // they touch, so it is enough to sort those (page, first slot, last slot) ranges and look
+        // for two that overlap in one page.
+        struct Range { int32_t page, lo, hi; };
+        std::vector<Range> touched;
+        for (int s = 0; s < B; ++s) {
+            const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
+            if (ql == 0) continue;
+            const int32_t *row = b->block_tables + (size_t)s * (size_t)b->table_stride;
+            for (int32_t p = cl - ql; p < cl;) {
+                const int32_t lp = p / kPageSize, last = std::min(cl, (lp + 1) * kPageSize) - 1;
+                touched.push_back({row[lp], p % kPageSize, last % kPageSize});
+                p = last + 1;
+            }
+        }
+        std::sort(touched.begin(), touched.end(), [](const Range &a, const Range &c) {
+            return a.page != c.page ? a.page < c.page : a.lo < c.lo;
+        });
+        for (size_t i = 1; i < touched.size(); ++i) {
+            if (touched[i].page != touched[i - 1].page) continue;
+            if (touched[i].lo <= touched[i - 1].hi) return AP_ERR_BAD_BLOCK_TABLE;
+            touched[i].hi = std::max(touched[i].hi, touched[i - 1].hi);
+        }
     }
 
     // ---- decode: cut the (row, kv head) page streams into per-CTA item lists
@@ -332,60 +351,64 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     std::vector<MergeEntry> merges;
     int n_slots = 0;
     if (decode_rows > 0) {
-        int64_t total_cost = 0;
+        // One pass with an adaptive share: each list gets (cost still to place) / (lists still to
+        // fill), so rounding cuts to stage boundaries and the extra items that cuts create spread over
+        // the lists that follow instead of piling up in a last one.  `left` counts pages plus
+        // kItemCost per item still to emit.
+        int64_t left = 0;
         for (int s = 0; s < B; ++s)
             if (b->q_lens[s] == 1)
-                total_cost += (int64_t)Hkv * (((int64_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize + kItemCost);
-        int64_t target = std::max<int64_t>((total_cost + max_ctas - 1) / max_ctas, 2 * kStage + kItemCost);
-        for (int attempt = 0; attempt < 64; ++attempt) {
-            items.clear(); cta_begin.clear(); merges.clear(); n_slots = 0;
-            cta_begin.push_back(0);
-            int64_t cap = target;
-            auto next_cta = [&]() {
-                if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
-                cap = target;
-            };
-            for (int s = 0; s < B; ++s) {
-                if (b->q_lens[s] != 1) continue;
-                const int32_t cl = b->ctx_lens[s];
-                const int32_t pages = (cl + kPageSize - 1) / kPageSize;
-                for (int g = 0; g < Hkv; ++g) {
-                    int32_t rem = pages, pb = 0;
-                    const size_t first = items.size();
-                    while (rem > 0) {
-                        int64_t avail = cap - kItemCost;
-                        if (avail < kStage && avail < rem) { next_cta(); continue; }
-                        int32_t take = (int32_t)std::min<int64_t>(rem, avail);
-                        if (take < rem) take = take / kStage * kStage;
-                        DecodeItem it{};
-                        it.q_row = row0[(size_t)s];
-                        it.kv_head = g;
-                        it.bt_offset = bt_off[(size_t)s];
-                        it.page_begin = pb;
-                        it.page_count = take;
-                        it.kv_len = cl;
-                        it.part_slot = -1;
-                        it.merge_index = -1;
-                        items.push_back(it);
-                        cap -= take + kItemCost;
-                        pb += take;
-                        rem -= take;
-                        if (cap < kItemCost + kStage) next_cta();
-                    }
-                    if (items.size() - first > 1) {
-                        MergeEntry m{row0[(size_t)s], g, n_slots, (int32_t)(items.size() - first)};
-                        merges.push_back(m);
-                        for (size_t i = first; i < items.size(); ++i) {
-                            items[i].part_slot = n_slots++;
-                            items[i].merge_index = (int32_t)merges.size() - 1;
-                        }
+                left += (int64_t)Hkv * (((int64_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize + kItemCost);
+        const int64_t min_share = 2 * kStage + kItemCost;
+        items.reserve((size_t)decode_rows * Hkv + 2 * (size_t)max_ctas);
+        cta_begin.reserve((size_t)max_ctas + 1);
+        cta_begin.push_back(0);
+        // (+ kStage: about what a list loses to rounding; without it the loss drifts to the last lists)
+        int64_t cap = std::max<int64_t>((left + max_ctas - 1) / max_ctas + kStage, min_share);
+        auto next_cta = [&]() {
+            if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
+            const int lists_left = max_ctas - ((int)cta_begin.size() - 1);
+            cap = lists_left <= 1 ? INT64_MAX / 2 : std::max<int64_t>((left + lists_left - 1) / lists_left + kStage, min_share);
+        };
+        for (int s = 0; s < B; ++s) {
+            if (b->q_lens[s] != 1) continue;
+            const int32_t cl = b->ctx_lens[s];
+            const int32_t pages = (cl + kPageSize - 1) / kPageSize;
+            for (int g = 0; g < Hkv; ++g) {
+                int32_t rem = pages, pb = 0;
+                const size_t first = items.size();
+                while (rem > 0) {
+                    int64_t avail = cap - kItemCost;
+                    if (avail < kStage && avail < rem) { next_cta(); continue; }
+                    int32_t take = (int32_t)std::min<int64_t>(rem, avail);
+                    if (take < rem) take = take / kStage * kStage;
+                    DecodeItem it{};
+                    it.q_row = row0[(size_t)s];
+                    it.kv_head = g;
+                    it.bt_offset = bt_off[(size_t)s];
+                    it.page_begin = pb;
+                    it.page_count = take;
+                    it.kv_len = cl;
+                    it.part_slot = -1;
+                    it.merge_index = -1;
+                    items.push_back(it);
+                    cap -= take + kItemCost;
+                    pb += take;
+                    rem -= take;
+                    left -= take + (rem > 0 ? 0 : kItemCost);   // a cut leaves one more item to emit
+                    if (cap < kItemCost + kStage) next_cta();
+                }
+                if (items.size() - first > 1) {
+                    MergeEntry m{row0[(size_t)s], g, n_slots, (int32_t)(items.size() - first)};
+                    merges.push_back(m);
+                    for (size_t i = first; i < items.size(); ++i) {
+                        items[i].part_slot = n_slots++;
+                        items[i].merge_index = (int32_t)merges.size() - 1;
                     }
                 }
             }
-            if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
-            if ((int)cta_begin.size() - 1 <= max_ctas) break;
-            target += std::max<int64_t>(1, target / 256);
         }
+        if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
     }
     const int n_ctas = cta_begin.empty() ? 0 : (int)cta_begin.size() - 1;
     // Inside a CTA, items of cut streams go first: their partials are then merged
@@ -651,17 +674,26 @@ int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, cons
     if (!pool || !batch) return AP_ERR_INVALID_ARG;
     if (pool->desc.device < 0) return AP_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    ap_plan *plan = nullptr;
-    int rc = ap_plan_create(&plan, pool, batch, stream);
-    if (rc != AP_OK) return rc;
-    const size_t n = (size_t)plan->info.n_new;
-    if (n == 0) { ap_plan_destroy(plan); return AP_OK; }
-    if (!q_host || !k_new_host || !v_new_host || !out_host) { ap_plan_destroy(plan); return AP_ERR_INVALID_ARG; }
+    if (batch->batch < 0 || batch->num_q_heads <= 0 || (batch->batch > 0 && !batch->q_lens)) return AP_ERR_INVALID_ARG;
+    // The input copies do not depend on the plan, so they are issued first and run while the host
+    // plans; only their sizes (the number of new tokens) are needed up front.
+    size_t n = 0;
+    for (int s = 0; s < batch->batch; ++s) {
+        if (batch->q_lens[s] < 0) return AP_ERR_INVALID_ARG;
+        n += (size_t)batch->q_lens[s];
+    }
+    if (n > (size_t)1 << 30) return AP_ERR_UNSUPPORTED;
+    if (n > 0 && (!q_host || !k_new_host || !v_new_host || !out_host)) return AP_ERR_INVALID_ARG;
     DeviceGuard guard(pool->desc.device);
-    if (!guard.ok) { ap_plan_destroy(plan); return AP_ERR_CUDA; }
+    if (!guard.ok) return AP_ERR_CUDA;
     const size_t d = (size_t)pool->desc.head_dim, Hq = (size_t)batch->num_q_heads, Hkv = (size_t)pool->desc.num_kv_heads;
+    if (Hq % Hkv != 0 || Hq / Hkv > 8) return Hq % Hkv != 0 ? AP_ERR_INVALID_ARG : AP_ERR_UNSUPPORTED;
     const size_t q_bytes = align_up(n * Hq * d * 2, 256), kv_bytes = align_up(n * Hkv * d * 2, 256);
-    const size_t lse_bytes = align_up(n * Hq * 4, 256), ws_bytes = align_up(plan->ws.bytes, 256);
+    const size_t lse_bytes = align_up(n * Hq * 4, 256);
+    // every decode CTA leaves at most two partials, which bounds the workspace before planning
+    const size_t max_slots = 2 * (size_t)std::max(1, pool->sm_count * decode_ctas_per_sm((int)d));
+    const size_t ws_bytes = align_up(max_slots * (Hq / Hkv) * d * sizeof(float), 256) +
+                            align_up(max_slots * (Hq / Hkv) * sizeof(float), 256);
     const size_t total = 2 * q_bytes + 2 * kv_bytes + lse_bytes + ws_bytes;
     if (total > pool->stage_bytes) {
         if (pool->stage_dev) {
@@ -673,7 +705,6 @@ int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, cons
         const size_t want = total + total / 4;
         if (cudaMalloc(&pool->stage_dev, want) != cudaSuccess) {
             (void)cudaGetLastError();
-            ap_plan_destroy(plan);
             return AP_ERR_CUDA;
         }
         pool->stage_bytes = want;
@@ -682,17 +713,28 @@ int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, cons
     void *dq = base, *dout = base + q_bytes, *dk = base + 2 * q_bytes, *dv = base + 2 * q_bytes + kv_bytes;
     float *dlse = (float *)(base + 2 * q_bytes + 2 * kv_bytes);
     void *dws = base + 2 * q_bytes + 2 * kv_bytes + lse_bytes;
-    bool ok = cudaMemcpyAsync(dq, q_host, n * Hq * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
-              cudaMemcpyAsync(dk, k_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
-              cudaMemcpyAsync(dv, v_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (ok) {
-        rc = ap_kv_append(pool, plan, dk, dv, stream);
-        if (rc == AP_OK) rc = ap_attention_iteration(pool, plan, dq, dout, dlse, dws, ws_bytes, stream);
-        if (rc == AP_OK) {
-            ok = cudaMemcpyAsync(out_host, dout, n * Hq * d * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-            if (ok && lse_host)
-                ok = cudaMemcpyAsync(lse_host, dlse, n * Hq * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-        }
+    bool ok = n == 0 ||
+              (cudaMemcpyAsync(dq, q_host, n * Hq * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+               cudaMemcpyAsync(dk, k_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+               cudaMemcpyAsync(dv, v_new_host, n * Hkv * d * 2, cudaMemcpyHostToDevice, st) == cudaSuccess);
+    if (!ok) {
+        (void)cudaGetLastError();
+        return AP_ERR_CUDA;
+    }
+    ap_plan *plan = nullptr;
+    int rc = ap_plan_create(&plan, pool, batch, stream);
+    if (rc != AP_OK) {               // the copies already queued only touch the staging buffer,
+        (void)cudaStreamSynchronize(st);   // but they read the caller's memory: let them finish
+        return rc;
+    }
+    if (n == 0) { ap_plan_destroy(plan); return AP_OK; }
+    if (plan->ws.bytes > ws_bytes) { ap_plan_destroy(plan); return AP_ERR_WORKSPACE_TOO_SMALL; }
+    rc = ap_kv_append(pool, plan, dk, dv, stream);
+    if (rc == AP_OK) rc = ap_attention_iteration(pool, plan, dq, dout, dlse, dws, ws_bytes, stream);
+    if (rc == AP_OK) {
+        ok = cudaMemcpyAsync(out_host, dout, n * Hq * d * 2, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        if (ok && lse_host)
+            ok = cudaMemcpyAsync(lse_host, dlse, n * Hq * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
     }
     if (!ok) { (void)cudaGetLastError(); rc = AP_ERR_CUDA; }
     const int dev_status = ap_last_device_status(pool, stream);  // synchronises the stream
