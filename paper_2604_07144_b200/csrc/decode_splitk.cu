@@ -224,6 +224,11 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
     }
     __syncthreads();
     auto get_item = [&](int it) -> DecodeItem { return it - item_begin < kSmemItems ? s_items[it - item_begin] : items[it]; };
+    // Everything up to here reads only the plan (uploaded before the step's kernels), so it may
+    // overlap the tail of the kernel before this one; the pool, q, the partial buffers and the
+    // counters may not be touched before that kernel is done.
+    griddep_launch_dependents();
+    if (warp != kConsumerWarps) griddep_wait();
 
     int stage = 0;
     uint32_t phase = 0;
@@ -236,6 +241,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         }
         DecodeItem item = get_item(item_begin);
         int32_t cur = lane < item.page_count ? __ldg(bt_flat + item.bt_offset + item.page_begin + lane) : 0;
+        griddep_wait();      // after the first block-table entries are on their way
         for (int it = item_begin; it < item_end; ++it) {
             const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
             const int npages = item.page_count;
@@ -544,11 +550,12 @@ cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const v
         configured[dev] = true;
     }
     const float scale_log2 = plan->scale * 1.4426950408889634f;
-    decode_splitk_kernel<D><<<(unsigned)plan->info.decode_ctas, kDecodeThreads, Cfg::kSmemBytes, stream>>>(
-        pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
-        plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, plan->group,
-        pool->desc.num_pages, scale_log2, pool->d_status);
-    return cudaGetLastError();
+    cudaError_t e = launch_overlapped(
+        decode_splitk_kernel<D>, (unsigned)plan->info.decode_ctas, (unsigned)kDecodeThreads, (size_t)Cfg::kSmemBytes,
+        stream, pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
+        plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads,
+        plan->group, pool->desc.num_pages, scale_log2, pool->d_status);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

@@ -128,6 +128,25 @@ cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, co
 cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                            float *lse, cudaStream_t stream);
 
+// Launch with programmatic stream serialization: the kernel may begin (up to its griddep_wait)
+// before the previous kernel in the stream has drained, which hides launch latency and preamble.
+// Every kernel launched this way touches data written by earlier work only after griddep_wait.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                                     cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Decode kernel launch geometry (used by the planner to size the item lists).
 int decode_ctas_per_sm(int head_dim);
 constexpr int kDecodePagesPerStage = 4;

@@ -2,6 +2,7 @@
 // pool.  A pure 16-byte-vector copy, so the result is bit-exact by
 // construction.  HBM-bound and small next to attention.
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace ap {
 
@@ -22,7 +23,9 @@ __global__ void __launch_bounds__(256) kv_append_kernel(uint4 *__restrict__ k_po
     const int64_t rh = v / chunks_per_row;
     const int g = (int)(rh % num_kv_heads);
     const int64_t row = rh / num_kv_heads;
-    const int32_t dst = __ldg(append_dst + row);
+    const int32_t dst = __ldg(append_dst + row);      // plan data: uploaded before any kernel of the step
+    ptx::griddep_launch_dependents();
+    ptx::griddep_wait();                              // the pool may still be read by the kernel before
     const int32_t page = dst >> 4, slot = dst & 15;
     if (page < 0 || page >= num_pages) {
         atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
@@ -41,10 +44,11 @@ cudaError_t launch_kv_append(const ap_kv_pool *pool, const ap_plan *plan, const 
     const int64_t n_vec = plan->info.n_new * pool->desc.num_kv_heads * chunks;
     const int threads = 256;
     const int64_t blocks = (n_vec + threads - 1) / threads;
-    kv_append_kernel<<<(unsigned)blocks, threads, 0, stream>>>(
-        (uint4 *)pool->desc.k_base, (uint4 *)pool->desc.v_base, (const uint4 *)k_new, (const uint4 *)v_new,
-        plan->d_append_dst, n_vec, pool->desc.num_kv_heads, chunks, pool->desc.num_pages, pool->d_status);
-    return cudaGetLastError();
+    cudaError_t e = launch_overlapped(kv_append_kernel, (unsigned)blocks, (unsigned)threads, 0, stream,
+                                      (uint4 *)pool->desc.k_base, (uint4 *)pool->desc.v_base, (const uint4 *)k_new,
+                                      (const uint4 *)v_new, plan->d_append_dst, n_vec, pool->desc.num_kv_heads, chunks,
+                                      pool->desc.num_pages, pool->d_status);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace ap

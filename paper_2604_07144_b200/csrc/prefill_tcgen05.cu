@@ -173,6 +173,10 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // The preamble above reads only the plan; q, the pool and the outputs wait for the kernel
+    // before this one in the stream.
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
@@ -450,10 +454,12 @@ cudaError_t launch_prefill_t(const ap_kv_pool *pool, const ap_plan *plan, const 
     CUtensorMap q_map;
     if (encode_q_tensor_map(&q_map, q, plan->info.n_new, plan->num_q_heads, D) != AP_OK) return cudaErrorInvalidValue;
     const float scale_log2 = plan->scale * 1.4426950408889634f;
-    prefill_tcgen05_kernel<D><<<(unsigned)plan->info.prefill_tiles, kPrefillThreads, Cfg::kSmemBytes, stream>>>(
-        q_map, pool->k_map, pool->v_map, plan->d_tiles, plan->d_bt_flat, (__nv_bfloat16 *)out, lse,
-        plan->num_q_heads, pool->desc.num_kv_heads, pool->desc.num_pages, scale_log2, pool->d_status);
-    return cudaGetLastError();
+    cudaError_t e = launch_overlapped(
+        prefill_tcgen05_kernel<D>, (unsigned)plan->info.prefill_tiles, (unsigned)kPrefillThreads,
+        (size_t)Cfg::kSmemBytes, stream, q_map, pool->k_map, pool->v_map, plan->d_tiles, plan->d_bt_flat,
+        (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, pool->desc.num_pages, scale_log2,
+        pool->d_status);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

@@ -22,6 +22,15 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 
 // make barrier initialisation visible to the async proxy (TMA, tcgen05.commit)
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start while the kernel before it in the stream is still running.  `griddep_wait` blocks
+// until that kernel has completed and its writes are visible (a no-op without the attribute);
+// `griddep_launch_dependents` lets the kernel after this one start its own preamble early.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
