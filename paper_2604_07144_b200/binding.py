@@ -27,7 +27,8 @@ AP_ERR_TIMEOUT = -6
 AP_ERR_UNSUPPORTED = -7
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libap_serving.so")
+#: the shared library; ``AP_SERVING_LIB`` selects another build of the same ABI
+LIB_PATH = os.environ.get("AP_SERVING_LIB") or os.path.join(_HERE, "libap_serving.so")
 
 #: every symbol ``include/ap_serving.h`` declares
 EXPORTED_SYMBOLS = (

@@ -14,7 +14,7 @@
 //               of the second product, rescale O in TMEM when the running max has
 //               moved enough, and write the normalised output at the end
 //   warp 8      producer: Q tiles once, then K and V tiles into one 5-slot ring
-//   warp 9      MMA issuer: S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
+//   warp 9      MMA issuer (converged warp, one elected lane issues): S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
 //               tensor pipe works on one tile while the other tile's softmax runs
 //   warps 10-11 idle (they only complete the third warpgroup for the register split)
 //
@@ -222,7 +222,9 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             }
         } else if (warp == kMmaWarp) {
             // ------------------------------------------------ MMA issuer --
-            if (lane == 0) {
+            // The warp runs this block converged; `leader` selects the lane that issues.
+            {
+                const uint32_t leader = elect_one();
                 constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
                 constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
                 bool ok = wait_or_abort(q_full, 0, abort_flag);
@@ -243,10 +245,10 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     const uint32_t d = tmem + Cfg::kColS + x * 128;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss_w(d, a0 + (uint32_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4), q_hi,
+                        umma_ss(leader, d, a0 + (uint32_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4), q_hi,
                                   b0 + (uint32_t)(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), k_hi, kIdescQK,
                                   ks > 0 ? 1u : 0u);
-                    umma_commit(&s_full[x]);
+                    umma_commit(leader, &s_full[x]);
                 };
                 // O_x += P_x V with V in ring slot `slot`.  P: bf16 pairs in the first 64 columns of S_x
                 // (A operand from TMEM, 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
@@ -256,11 +258,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     if (!first_step) {
 #pragma unroll
                         for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts_w(d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV, 1u);
+                            umma_ts(leader, d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV, 1u);
                     } else {
 #pragma unroll
                         for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts_w(d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV,
+                            umma_ts(leader, d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV,
                                       ks > 0 ? 1u : 0u);
                     }
                 };
@@ -268,7 +270,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 if (ok) {
                     tcgen05_fence_after();
                     for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);     // K_0 is ring entry 0, slot 0
-                    umma_commit(&kv_empty[0]);
+                    umma_commit(leader, &kv_empty[0]);
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
                     const int nv = kv_seq_v(j, n_steps), nk = kv_seq_k(j + 1);
@@ -282,14 +284,14 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                                                          abort_flag)) { ok = false; break; }
                             issue_qk(x, nk % kKvSlots);                // overwrites S_x / P_x after the product above
                         } else {
-                            umma_commit(&o_done[x]);
+                            umma_commit(leader, &o_done[x]);
                         }
                     }
                     if (!ok) break;
-                    umma_commit(&kv_empty[nv % kKvSlots]);
-                    if (j + 1 < n_steps) umma_commit(&kv_empty[nk % kKvSlots]);
+                    umma_commit(leader, &kv_empty[nv % kKvSlots]);
+                    if (j + 1 < n_steps) umma_commit(leader, &kv_empty[nk % kKvSlots]);
                 }
-                if (!ok) {
+                if (!ok && leader) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                 }
@@ -369,8 +371,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         float2 xy = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i) & 31]),
                                                            __uint_as_float(sreg[2 * c + (i >> 4)][(2 * i + 1) & 31])),
                                                sc2, nms2);
-                        // every other pair goes to the FMA pipe instead of the special-function unit
-                        if (i & 1) {
+                        // one pair in four goes to the FMA pipe instead of the special-function unit
+                        if ((i & 3) == 3) {
                             xy = exp2_poly2(xy);
                         } else {
                             xy.x = exp2_approx(xy.x);
