@@ -42,8 +42,8 @@ UNIT = "KV-tokens/s"
 # bench workload (ncu capture summarised under profiles/), keyed by the hash of
 # the kernel's source file (decode_splitk.cu) the counters were taken from; a changed kernel reports null.
 NCU_TRAFFIC = {
-    # profiles/decode_splitk_config2.md: 537.0 MB read + 5.1 MB written per launch (algorithmic 535.0 MB)
-    (2, "d09a690fa3bb9edc"): 542.1e6,
+    # profiles/decode_splitk_config2.md: 536.9 MB read + 5.3 MB written per launch (algorithmic 535.0 MB)
+    (2, "04f79039326158ed"): 542.2e6,
 }
 
 
