@@ -318,6 +318,9 @@ def main():
     ap_.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
     ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
     ap_.add_argument("--no-cpu-baseline", action="store_true")
+    ap_.add_argument("--side-by-side", type=int, default=None,
+                     help="mixed iterations: 0 = decode then prefill, 1 = planner decides (library default), "
+                          "k >= 2 = decode on k CTAs next to prefill")
     args = ap_.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -361,6 +364,8 @@ def main():
         kp, vp = (k0, v0) if c == 0 else (k0.clone(), v0.clone())
         k_planes.append(kp); v_planes.append(vp)
         pools.append(ap.kv_pool_create(batch.num_pages, hkv, d, kp, vp, device=local_rank))
+        if args.side_by_side is not None:
+            ap.kv_pool_set_side_by_side(pools[-1], args.side_by_side)
         plans.append(ap.plan_create(pools[-1], batch.q_lens, batch.ctx_lens, batch.block_tables, hq))
     info = ap.plan_get_info(plans[0])
     q, k_new, v_new = dev_bf16(batch.q), dev_bf16(batch.k_new), dev_bf16(batch.v_new)
@@ -472,6 +477,18 @@ def main():
             "bytes_per_launch": alg["decode_kernel"], "us_per_launch": 1e3 * dec_ms / max(dec_n, 1),
             "frac_of_nominal_8TBs": achieved / 8000.0,
         }
+        if info["side_by_side"]:
+            roofline["note"] = (f"in this plan decode runs on {info['decode_ctas']} SMs next to the prefill kernel, so its own "
+                                "time is not a whole-GPU bandwidth figure; see step_roofline")
+        # whole step against the slower of its two bounds: all algorithmic bytes at the measured copy
+        # bandwidth, all algorithmic flops at the measured bf16 peak
+        t_bytes = alg["total"] / (peaks["hbm_gbs"] * 1e9)
+        t_flops = (alg["decode_flops"] + alg["prefill_flops"]) / (peaks["bf16_tflops"] * 1e12)
+        step_roofline = {"bound_us": max(t_bytes, t_flops) * 1e6, "bytes_us": t_bytes * 1e6, "flops_us": t_flops * 1e6,
+                         "sum_us": (t_bytes + t_flops) * 1e6, "step_us": ms_per_step * 1e3,
+                         "frac": max(t_bytes, t_flops) / (ms_per_step * 1e-3),
+                         "note": "bound = max(bytes / copy bandwidth, flops / bf16 peak): reachable only if the "
+                                 "HBM-bound and the tensor-bound parts overlap perfectly; sum = no overlap"}
         kernels = {name: {"launches": n, "us_per_launch": (1e3 * ms / n if n else None)} for name, (ms, n) in kt.items()}
         res = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -488,8 +505,9 @@ def main():
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
                     "includes": "plan build + upload, H2D of q/k_new/v_new, append, attention, D2H of out/lse, sync"},
             "plan": {"host_ms": plan_ms, "in_value": False, "in_e2e": True, **{k: info[k] for k in (
-                "decode_items", "decode_ctas", "merge_entries", "prefill_tiles")}},
+                "decode_items", "decode_ctas", "merge_entries", "prefill_tiles", "side_by_side")}},
             "roofline": roofline,
+            "step_roofline": step_roofline,
             "kernels": kernels,
             "kernel_timing": {"how": "second pass of the same K steps with a CUDA-event pair around every kernel, "
                                      "right after the timed pass; the timed pass itself has no events between kernels",

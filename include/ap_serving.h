@@ -102,6 +102,20 @@ int ap_kv_pool_destroy(ap_kv_pool *pool);
 void *ap_kv_pool_k_base(const ap_kv_pool *pool);
 void *ap_kv_pool_v_base(const ap_kv_pool *pool);
 
+/*
+ * Side-by-side execution of mixed iterations (Sec. 5.3: the batch an iteration
+ * runs, prefill chunks next to decode tokens, is what the scheduling policy
+ * composes).  When a plan holds both decode rows and prefill chunks, the decode
+ * kernel can be confined to k persistent CTAs on the caller's stream while the
+ * prefill kernel runs at the same time on a stream the pool owns (joined back
+ * into the caller's stream before ap_attention_iteration returns control of it).
+ * mode 0: never; mode 1 (default): ap_plan_create decides per plan from a cost
+ * model and picks k; mode >= 2: always, with k = mode decode CTAs (clamped).
+ * Applies to plans created afterwards; results are identical in every mode.
+ * ap_plan_info.side_by_side reports what a plan does.  mode < 0 -> INVALID_ARG.
+ */
+int ap_kv_pool_set_side_by_side(ap_kv_pool *pool, int32_t mode);
+
 /* Host page allocator (per-request page ownership; pages are relocatable units,
  * Sec. 4.1 Phase 2).  alloc is all-or-nothing: OUT_OF_PAGES leaves the free
  * list unchanged.  out_ids / ids: host.  free of a page that is not allocated,
@@ -158,6 +172,7 @@ typedef struct ap_plan_info {
     int64_t prefill_tiles;   /* work units of the prefill kernel */
     int64_t launches_append; /* kernels ap_kv_append launches for this plan */
     int64_t launches_attention; /* kernels ap_attention_iteration launches for this plan */
+    int64_t side_by_side;    /* 1 if the decode and prefill kernels of this plan run concurrently */
 } ap_plan_info;
 int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
 

@@ -34,7 +34,7 @@ LIB_PATH = os.environ.get("AP_SERVING_LIB") or os.path.join(_HERE, "libap_servin
 EXPORTED_SYMBOLS = (
     "ap_status_string", "ap_kv_pool_bytes", "ap_kv_pool_create", "ap_kv_pool_destroy",
     "ap_kv_pool_k_base", "ap_kv_pool_v_base", "ap_kv_pool_alloc_pages", "ap_kv_pool_free_pages",
-    "ap_kv_pool_seed_free_list", "ap_kv_pool_num_free", "ap_plan_create", "ap_plan_destroy",
+    "ap_kv_pool_seed_free_list", "ap_kv_pool_num_free", "ap_kv_pool_set_side_by_side", "ap_plan_create", "ap_plan_destroy",
     "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append",
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
@@ -64,7 +64,8 @@ class BatchDesc(ctypes.Structure):
 class PlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "n_new", "kv_tokens", "decode_rows", "prefill_seqs", "prefill_pairs", "decode_items",
-        "decode_ctas", "merge_entries", "prefill_tiles", "launches_append", "launches_attention")]
+        "decode_ctas", "merge_entries", "prefill_tiles", "launches_append", "launches_attention",
+        "side_by_side")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -108,6 +109,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_kv_pool_free_pages": (ctypes.c_int, [vp, i32, vp]),
         "ap_kv_pool_seed_free_list": (ctypes.c_int, [vp, u64]),
         "ap_kv_pool_num_free": (i32, [vp]),
+        "ap_kv_pool_set_side_by_side": (ctypes.c_int, [vp, i32]),
         "ap_plan_create": (ctypes.c_int, [ctypes.POINTER(vp), vp, ctypes.POINTER(BatchDesc), vp]),
         "ap_plan_destroy": (ctypes.c_int, [vp]),
         "ap_plan_workspace_bytes": (sz, [vp]),
@@ -224,6 +226,11 @@ def kv_pool_free_pages(pool: KVPool, ids: Sequence[int]) -> None:
 
 def kv_pool_seed_free_list(pool: KVPool, seed: int) -> None:
     _check(load().ap_kv_pool_seed_free_list(pool.handle, seed), "ap_kv_pool_seed_free_list")
+
+
+def kv_pool_set_side_by_side(pool: KVPool, mode: int) -> None:
+    """0: never run decode and prefill concurrently; 1: per-plan decision (default); k >= 2: always, k decode CTAs."""
+    _check(load().ap_kv_pool_set_side_by_side(pool.handle, int(mode)), "ap_kv_pool_set_side_by_side")
 
 
 def kv_pool_num_free(pool: KVPool) -> int:

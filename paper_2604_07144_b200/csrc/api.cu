@@ -84,6 +84,53 @@ cudaEvent_t take_event(ap_kv_pool *pool) {
     return e;
 }
 
+// Side-by-side execution of a mixed iteration.  Decode is bound by HBM when it has the whole GPU
+// (~41 GB/s per SM at 148 SMs) but one SM's decode pipeline sustains more (~58 GB/s: its ring keeps
+// about 68 KB in flight over a ~1.1 us memory latency), while prefill is bound by the SMs it has.
+// So decode is confined to k SMs, where it is SM-bound, and prefill runs on the others at the same
+// time; the iteration then takes about (W_d + W_p) / #SM, with W the SM-time of each part.  k is
+// the smallest count that lets decode finish within 85 % of that time; beyond ~0.7 #SM decode would
+// be HBM-bound again and nothing is gained, so the plan stays sequential.  The constants were
+// measured on B200 with the 8B attention shape.  Returns 0 for "sequential".
+constexpr double kDecodeSmGBs = 58.0;        // GB/s of KV one SM's decode pipeline sustains
+constexpr double kDecodeGpuGBs = 6000.0;     // GB/s decode reaches with all SMs
+constexpr double kPrefillStepUs = 2.1;       // one 128-key step of a two-tile unit at d = 128
+constexpr double kPrefillStepSingleUs = 1.5; // the same for a one-tile unit
+constexpr double kPrefillUnitUs = 5.3;       // prologue + epilogue + relaunch gap of a unit
+
+int side_by_side_decode_ctas(const ap_kv_pool *pool, const ap_batch_desc *b, int d, int Hkv, int G, int max_ctas) {
+    const int mode = pool->side_by_side_mode;
+    if (mode == 0) return 0;
+    double decode_bytes = 0.0, w_p = 0.0;
+    int64_t decode_rows = 0, prefill_seqs = 0;
+    const double d_scale = (double)d / 128.0;
+    for (int s = 0; s < b->batch; ++s) {
+        const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
+        if (ql == 1) {
+            ++decode_rows;
+            decode_bytes += (double)((cl + kPageSize - 1) / kPageSize) * kPageSize * Hkv * d * 4.0;
+        } else if (ql > 1) {
+            ++prefill_seqs;
+            for (int32_t t0 = 0; t0 < ql; t0 += 128) {
+                const int steps = (cl - ql + t0 + std::min(128, ql - t0) + 127) / 128;
+                const int pairs = G / 2, singles = G % 2;
+                w_p += (double)Hkv * (pairs * (steps * kPrefillStepUs * d_scale + kPrefillUnitUs) +
+                                      singles * (steps * kPrefillStepSingleUs * d_scale + kPrefillUnitUs));
+            }
+        }
+    }
+    if (decode_rows == 0 || prefill_seqs == 0) return 0;
+    if (mode >= 2) return std::min(mode, max_ctas);
+    const int sms = pool->sm_count;
+    const double w_d = decode_bytes / (kDecodeSmGBs * 1e3);              // SM-microseconds
+    const double t_serial = decode_bytes / (kDecodeGpuGBs * 1e3) + w_p / sms;
+    const double t_side = (w_d + w_p) / sms;
+    if (t_serial - t_side < 10.0 || t_serial - t_side < 0.05 * t_serial) return 0;
+    const int k = (int)std::ceil(w_d / (0.85 * t_side));
+    if (k < 8 || k > (7 * sms) / 10 || k >= max_ctas) return 0;
+    return k;
+}
+
 // Brackets one kernel launch with events when profiling is on.
 struct TimedScope {
     ap_kv_pool *pool;
@@ -180,6 +227,16 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
             rc = AP_ERR_CUDA;
             break;
         }
+        {
+            int least = 0, greatest = 0;
+            if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess ||
+                cudaStreamCreateWithPriority(&p->side_stream, cudaStreamNonBlocking, least) != cudaSuccess ||
+                cudaEventCreateWithFlags(&p->fork_event, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&p->join_event, cudaEventDisableTiming) != cudaSuccess) {
+                rc = AP_ERR_CUDA;
+                break;
+            }
+        }
         rc = encode_pool_tensor_map(&p->k_map, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
         if (rc != AP_OK) break;
         rc = encode_pool_tensor_map(&p->v_map, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
@@ -205,6 +262,9 @@ int ap_kv_pool_destroy(ap_kv_pool *pool) {
     for (auto &b : pool->plan_buffers) release_plan_buffer(b);
     for (auto &t : pool->timed) { (void)cudaEventDestroy(t.start); (void)cudaEventDestroy(t.stop); }
     for (auto &e : pool->spare_events) (void)cudaEventDestroy(e);
+    if (pool->side_stream) (void)cudaStreamDestroy(pool->side_stream);
+    if (pool->fork_event) (void)cudaEventDestroy(pool->fork_event);
+    if (pool->join_event) (void)cudaEventDestroy(pool->join_event);
     if (pool->stage_dev) (void)cudaFree(pool->stage_dev);
     if (pool->d_status) (void)cudaFree(pool->d_status);
     if (pool->owns_planes) {
@@ -213,6 +273,12 @@ int ap_kv_pool_destroy(ap_kv_pool *pool) {
     }
     (void)cudaGetLastError();
     delete pool;
+    return AP_OK;
+}
+
+int ap_kv_pool_set_side_by_side(ap_kv_pool *pool, int32_t mode) {
+    if (!pool || mode < 0) return AP_ERR_INVALID_ARG;
+    pool->side_by_side_mode = mode;
     return AP_OK;
 }
 
@@ -343,7 +409,9 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     }
 
     // ---- decode: cut the (row, kv head) page streams into per-CTA item lists
-    const int max_ctas = std::max(1, pool->sm_count * decode_ctas_per_sm(d));
+    int max_ctas = std::max(1, pool->sm_count * decode_ctas_per_sm(d));
+    const int side_ctas = side_by_side_decode_ctas(pool, b, (int)d, (int)Hkv, G, max_ctas);
+    if (side_ctas > 0) max_ctas = side_ctas;
     constexpr int kItemCost = 2;          // fixed per-item cost, in page units
     constexpr int kStage = kDecodePagesPerStage;
     std::vector<DecodeItem> items;
@@ -532,6 +600,8 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     info.prefill_tiles = (int64_t)tiles.size();
     info.launches_append = n_new > 0 ? 1 : 0;
     info.launches_attention = (items.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
+    plan->side_by_side = side_ctas > 0 && !items.empty() && !tiles.empty();
+    info.side_by_side = plan->side_by_side ? 1 : 0;
     *out = plan;
     return AP_OK;
 }
@@ -594,13 +664,31 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
     float *o_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.o_part_off) : nullptr;
     float *lse_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.lse_part_off) : nullptr;
     cudaError_t e = cudaSuccess;
-    if (plan->info.decode_items > 0) {
-        TimedScope timed(pool, AP_KERNEL_DECODE, st);
-        e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-    }
-    if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
-        TimedScope timed(pool, AP_KERNEL_PREFILL, st);
-        e = launch_prefill(pool, plan, q, out, lse, st);
+    if (plan->side_by_side) {
+        // Decode goes first, on the caller's stream, so that its few CTAs are resident when the
+        // prefill kernel's units (second stream, lower priority) fill the remaining SMs; as decode
+        // CTAs retire, prefill units take their SMs too.  The caller's stream continues after both.
+        e = cudaEventRecord(pool->fork_event, st);
+        if (e == cudaSuccess) {
+            TimedScope timed(pool, AP_KERNEL_DECODE, st);
+            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+        }
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pool->side_stream, pool->fork_event, 0);
+        if (e == cudaSuccess) {
+            TimedScope timed(pool, AP_KERNEL_PREFILL, pool->side_stream);
+            e = launch_prefill(pool, plan, q, out, lse, pool->side_stream);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(pool->join_event, pool->side_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, pool->join_event, 0);
+    } else {
+        if (plan->info.decode_items > 0) {
+            TimedScope timed(pool, AP_KERNEL_DECODE, st);
+            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+        }
+        if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
+            TimedScope timed(pool, AP_KERNEL_PREFILL, st);
+            e = launch_prefill(pool, plan, q, out, lse, st);
+        }
     }
     if (e != cudaSuccess) {
         (void)cudaGetLastError();

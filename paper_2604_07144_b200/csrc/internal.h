@@ -92,6 +92,11 @@ struct ap_kv_pool {
     // staging for ap_serving_iteration_host
     void *stage_dev = nullptr;
     size_t stage_bytes = 0;
+    // Side-by-side execution of mixed iterations: a low-priority second stream for the prefill
+    // kernel and the fork / join events that tie it to the caller's stream.
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t fork_event = nullptr, join_event = nullptr;
+    int side_by_side_mode = 1;        // 0 never, 1 decided per plan, >= 2 that many decode CTAs
     // per-kernel event timing (diagnostics)
     bool profiling = false;
     std::vector<ap::TimedLaunch> timed;
@@ -108,6 +113,7 @@ struct ap_plan {
     ap_plan_layout layout{};
     std::vector<int32_t> blob;   // host copy of the uploaded work lists
     int n_part_slots = 0;
+    bool side_by_side = false;   // decode on the caller's stream and prefill on the pool's second stream, concurrently
     ap::WorkspaceLayout ws{};
     // device pointers into buf.dev
     const int32_t *d_append_dst = nullptr;

@@ -25,7 +25,7 @@ def to_bits(t) -> np.ndarray:
 class GpuRun:
     """Pool + plan + device tensors of one batch."""
 
-    def __init__(self, batch: W.Batch, device: int = 0, scale: float = 0.0):
+    def __init__(self, batch: W.Batch, device: int = 0, scale: float = 0.0, side_by_side=None):
         import torch
         self.torch = torch
         self.batch = batch
@@ -41,6 +41,8 @@ class GpuRun:
                               device=dev)
         self.pool = ap.kv_pool_create(batch.num_pages, batch.num_kv_heads, batch.head_dim, self.k_pool,
                                       self.v_pool, device=device)
+        if side_by_side is not None:
+            ap.kv_pool_set_side_by_side(self.pool, side_by_side)
         self.plan = ap.plan_create(self.pool, batch.q_lens, batch.ctx_lens, batch.block_tables,
                                    batch.num_q_heads, softmax_scale=scale)
         self.info = ap.plan_get_info(self.plan)
@@ -80,9 +82,9 @@ def compare_outputs(out_bits: np.ndarray, lse: np.ndarray, ref_out: np.ndarray, 
     return float(err), float(lerr)
 
 
-def check_batch_full(batch: W.Batch, scale: float = 0.0):
+def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None):
     """Append + attention on the GPU against the oracle, every element."""
-    run = GpuRun(batch, scale=scale)
+    run = GpuRun(batch, scale=scale, side_by_side=side_by_side)
     try:
         run.append()
         run.attend()

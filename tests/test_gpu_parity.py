@@ -60,6 +60,36 @@ def test_mixed_ragged_small():
     check_batch_full(W.random_ragged(204, shape=W.SHAPE_8B, batch=5, max_ctx=900, max_q=300))
 
 
+@pytest.mark.parametrize("mode", [0, 3, 20])
+def test_mixed_iteration_side_by_side_modes(mode):
+    """Decode confined to a few CTAs on the caller's stream while prefill runs on the pool's second
+    stream (forced), and the sequential dispatch (mode 0): same results against the oracle, twice in
+    a row on the same pool (its stream and fork / join events are reused)."""
+    import oracle
+    from harness import compare_outputs, oracle_pools
+    batch = W._assemble("mixed_side_by_side", W.SHAPE_8B, W.make_rng(31),
+                        np.array([200, 1, 1, 1, 130, 1], np.int32),
+                        np.array([700, 333, 1500, 16, 130, 2049], np.int32), 1.3)
+    run = GpuRun(batch, side_by_side=mode)
+    try:
+        assert run.info["side_by_side"] == (1 if mode else 0)
+        if mode:
+            assert run.info["decode_ctas"] <= mode
+        run.append()
+        k_ref, v_ref = oracle_pools(batch)
+        ref_out, ref_lse = oracle.attention(k_ref, v_ref, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.q)
+        for _ in range(2):
+            run.out.fill_(float("nan"))
+            run.lse.fill_(float("nan"))
+            run.attend()
+            assert run.status() == 0
+            compare_outputs(to_bits(run.out)[:batch.n_new], run.lse.cpu().numpy()[:batch.n_new], ref_out, ref_lse,
+                            f"mode {mode}")
+        assert np.array_equal(to_bits(run.k_pool), k_ref) and np.array_equal(to_bits(run.v_pool), v_ref)
+    finally:
+        run.close()
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]

@@ -94,11 +94,13 @@ def test_plan_validation():
     ap.kv_pool_destroy(pool)
 
 
-def check_plan_coverage(batch: W.Batch):
+def check_plan_coverage(batch: W.Batch, side_by_side=None):
     """Every (decode row, kv head, page) appears in exactly one item; merge
     entries and part slots are consistent; every prefill row/head is in one tile."""
     hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
     pool = ap.kv_pool_create(batch.num_pages, hkv, d, device=-1)
+    if side_by_side is not None:
+        ap.kv_pool_set_side_by_side(pool, side_by_side)
     plan = ap.plan_create(pool, batch.q_lens, batch.ctx_lens, batch.block_tables, hq)
     ex = ap.plan_export(plan)
     info = ex["info"]
@@ -187,6 +189,28 @@ def test_plan_coverage_full_size_configs():
     assert i3["prefill_seqs"] == 8 and i3["decode_rows"] == 120 and i3["prefill_tiles"] == 8 * 4 * 16
     i4 = check_plan_coverage(W.config4(with_pool=False))
     assert i4["decode_ctas"] == 148 and i4["merge_entries"] > 0
+
+
+def test_side_by_side_planning():
+    """Mixed iterations: the planner confines decode to k CTAs (cost model or forced) and the
+    work lists still cover everything; pure decode / pure prefill plans stay sequential."""
+    b3 = W.config3(with_pool=False)
+    auto = check_plan_coverage(b3)                               # mode 1 is the default
+    assert auto["side_by_side"] == 1 and 48 <= auto["decode_ctas"] <= 96
+    off = check_plan_coverage(b3, side_by_side=0)
+    assert off["side_by_side"] == 0 and off["decode_ctas"] == 148
+    forced = check_plan_coverage(b3, side_by_side=40)
+    assert forced["side_by_side"] == 1 and forced["decode_ctas"] <= 40
+    assert forced["decode_items"] >= off["decode_rows"] * 8
+    for b in (W.config2(with_pool=False), W.config4(with_pool=False)):
+        assert check_plan_coverage(b, side_by_side=64)["side_by_side"] == 0
+    # a mixed batch too small to gain anything stays sequential under the cost model
+    small = W.random_ragged(5, batch=6, max_ctx=900, max_q=300)
+    assert check_plan_coverage(small)["side_by_side"] == 0
+    pool = host_pool()
+    with pytest.raises(ap.ApError):
+        ap.kv_pool_set_side_by_side(pool, -1)
+    ap.kv_pool_destroy(pool)
 
 
 def test_empty_batch_plans_to_nothing():
