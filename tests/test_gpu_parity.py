@@ -90,6 +90,48 @@ def test_mixed_iteration_side_by_side_modes(mode):
         run.close()
 
 
+@pytest.mark.parametrize("mode", [0, 3])
+def test_iteration_is_capturable_in_a_cuda_graph(mode):
+    """Append + attention issue no host synchronisation and take every buffer by address, so the
+    per-layer sequence of a model (here: the same layer four times) can be captured once into a CUDA
+    graph and replayed; with decode beside prefill the fork / join through the pool's second stream
+    is captured too.  The replayed result is checked against the oracle."""
+    import torch
+    import oracle
+    from harness import compare_outputs, oracle_pools
+    batch = W._assemble("graph_mixed", W.SHAPE_8B, W.make_rng(41), np.array([150, 1, 1, 1], np.int32),
+                        np.array([400, 90, 1300, 17], np.int32), 1.3)
+    run = GpuRun(batch, side_by_side=mode)
+    try:
+        assert run.info["side_by_side"] == (1 if mode else 0)
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            run.append()                       # warm-up outside the capture (first-launch attribute set-up)
+            run.attend()
+        stream.synchronize()
+        assert run.status() == 0
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for _ in range(4):
+                run.append()
+                run.attend()
+        k_ref, v_ref = oracle_pools(batch)
+        ref_out, ref_lse = oracle.attention(k_ref, v_ref, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.q)
+        for _ in range(2):
+            run.out.fill_(float("nan"))
+            run.lse.fill_(float("nan"))
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            assert run.status() == 0
+            compare_outputs(to_bits(run.out)[:batch.n_new], run.lse.cpu().numpy()[:batch.n_new], ref_out, ref_lse,
+                            f"graph replay, mode {mode}")
+        assert np.array_equal(to_bits(run.k_pool), k_ref) and np.array_equal(to_bits(run.v_pool), v_ref)
+        del graph
+    finally:
+        run.close()
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]
