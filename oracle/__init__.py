@@ -58,6 +58,7 @@ def bind(cdll: ctypes.CDLL) -> ctypes.CDLL:
     cdll.oracle_num_threads.restype = ctypes.c_int
     cdll.oracle_kv_append.restype = ctypes.c_int
     cdll.oracle_softmax_row.restype = ctypes.c_int
+    cdll.oracle_copy_pages.restype = ctypes.c_int
     for name in ("oracle_attention", "oracle_attention_samples", "oracle_merge_partials",
                  "oracle_attention_range"):
         getattr(cdll, name).restype = None
@@ -87,6 +88,20 @@ def kv_append(k_pool: np.ndarray, v_pool: np.ndarray, q_lens, ctx_lens, block_ta
         _p(k_pool), _p(v_pool), ctypes.c_int(num_pages), ctypes.c_int(hkv), ctypes.c_int(d),
         ctypes.c_int(len(q_lens)), _p(q_lens), _p(ctx_lens), _p(bt), ctypes.c_int(bt.shape[1]),
         _p(k_new), _p(v_new)))
+
+
+def copy_pages(k_dst: np.ndarray, v_dst: np.ndarray, k_src: np.ndarray, v_src: np.ndarray, dst_ids, src_ids) -> int:
+    """In place: page ``src_ids[i]`` of the source planes -> page ``dst_ids[i]`` of the destination
+    planes (all kv heads, K and V), simultaneously for all i.  The planes may be the same arrays."""
+    assert k_dst.flags.c_contiguous and v_dst.flags.c_contiguous
+    k_src, v_src = _u16(k_src), _u16(v_src)
+    assert k_dst.shape[1:] == k_src.shape[1:] and k_dst.shape[2] == 16
+    dst_ids, src_ids = _i32(dst_ids), _i32(src_ids)
+    assert len(dst_ids) == len(src_ids)
+    return int(lib().oracle_copy_pages(
+        _p(k_dst), _p(v_dst), ctypes.c_int(k_dst.shape[0]), _p(k_src), _p(v_src), ctypes.c_int(k_src.shape[0]),
+        ctypes.c_int(k_dst.shape[1]), ctypes.c_int(k_dst.shape[3]), ctypes.c_int(len(dst_ids)),
+        _p(dst_ids), _p(src_ids)))
 
 
 def attention(k_pool, v_pool, q_lens, ctx_lens, block_tables, q, scale: float = 0.0

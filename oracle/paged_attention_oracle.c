@@ -18,6 +18,8 @@
  *   append:    position p = ctx_len - q_len + t of sequence s lives in
  *              page  = block_table[s][p div 16], slot = p mod 16;
  *              K[page][kv_head][slot][:] <- k_new[row][kv_head][:]  (bit copy)
+ *   page copy: page src_ids[i] (all kv heads, K and V) -> page dst_ids[i], all
+ *              pairs at once (KV-cache migration between plans, Sec. 3.2)
  *   attention: query row (s,t), q head h, kv head g = h div (Hq/Hkv):
  *              x_j = scale * <q, k_j>  for j = 0..p   (causal bound j <= p)
  *              m = max_j x_j,  l = sum_j exp(x_j - m)
@@ -29,7 +31,9 @@
  * Pins (tests/test_oracle_pins.py): dense brute force on contiguous tensors,
  * softmax rows summing to 1, single-token context returning V, identical
  * keys returning the mean of V, q = 0 giving lse = ln(p+1), page-permutation
- * invariance, split/merge identity, chunking identity, append replay.
+ * invariance, split/merge identity, chunking identity, append replay; for the
+ * page copy: attention unchanged after moving every page to another pool and
+ * remapping the block tables, numpy's simultaneous gather/scatter, refusals.
  */
 #include <math.h>
 #include <stdint.h>
@@ -92,6 +96,43 @@ int oracle_kv_append(uint16_t *K, uint16_t *V, int num_pages, int Hkv, int d,
         }
     }
     return rc;
+}
+
+/*
+ * KV page copy (Sec. 3.2, Phase 2 "Reconfiguration": the transition between two
+ * plans migrates KV caches; a page is the unit that moves).  For i = 0..n-1 the
+ * whole page src_ids[i] of the source planes -- every kv head, every slot, both
+ * K and V -- is copied bit for bit to page dst_ids[i] of the destination
+ * planes.  All sources are read before any destination is written (the copies
+ * are simultaneous: a page may be both a source and another pair's
+ * destination), so the result does not depend on the order of the pairs.
+ * Returns 0, or -1 (nothing written) if an id is out of range or a destination
+ * appears twice.  The planes may be the same (copy inside one pool).
+ */
+int oracle_copy_pages(uint16_t *K_dst, uint16_t *V_dst, int num_pages_dst,
+                      const uint16_t *K_src, const uint16_t *V_src, int num_pages_src,
+                      int Hkv, int d, int n, const int32_t *dst_ids, const int32_t *src_ids)
+{
+    const size_t page_elems = (size_t)Hkv * ORACLE_PAGE * (size_t)d;
+    for (int i = 0; i < n; ++i) {
+        if (dst_ids[i] < 0 || dst_ids[i] >= num_pages_dst) return -1;
+        if (src_ids[i] < 0 || src_ids[i] >= num_pages_src) return -1;
+        for (int j = 0; j < i; ++j)
+            if (dst_ids[j] == dst_ids[i]) return -1;
+    }
+    if (n <= 0) return 0;
+    uint16_t *tmp = (uint16_t *)malloc(2 * (size_t)n * page_elems * sizeof(uint16_t));
+    if (!tmp) return -1;
+    for (int i = 0; i < n; ++i) {
+        memcpy(tmp + (2 * (size_t)i) * page_elems, K_src + (size_t)src_ids[i] * page_elems, page_elems * sizeof(uint16_t));
+        memcpy(tmp + (2 * (size_t)i + 1) * page_elems, V_src + (size_t)src_ids[i] * page_elems, page_elems * sizeof(uint16_t));
+    }
+    for (int i = 0; i < n; ++i) {
+        memcpy(K_dst + (size_t)dst_ids[i] * page_elems, tmp + (2 * (size_t)i) * page_elems, page_elems * sizeof(uint16_t));
+        memcpy(V_dst + (size_t)dst_ids[i] * page_elems, tmp + (2 * (size_t)i + 1) * page_elems, page_elems * sizeof(uint16_t));
+    }
+    free(tmp);
+    return 0;
 }
 
 /*

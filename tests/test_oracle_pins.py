@@ -217,10 +217,56 @@ def pin_append_replay():
     assert np.array_equal(k, b.k_pool)
 
 
+def pin_page_copy_migration():
+    """Page copy: (1) moving every used page of a batch into another pool and remapping the block
+    tables leaves attention bit-identical, the source pool and the unused destination pages untouched;
+    (2) it equals numpy's simultaneous gather/scatter, also for a rotation of pages inside one pool;
+    (3) bad ids and repeated destinations are refused without writing."""
+    b = W.random_ragged(61, batch=6, max_ctx=150, max_q=5)
+    k, v = _post_append(b)
+    o_ref, l_ref = oracle.attention(k, v, b.q_lens, b.ctx_lens, b.block_tables, b.q)
+    used = sorted({int(b.block_tables[s, i]) for s in range(b.batch) for i in range((int(b.ctx_lens[s]) + 15) // 16)})
+    rng = np.random.default_rng(7)
+    n_dst = b.num_pages + 11
+    new_of = dict(zip(used, rng.permutation(n_dst)[:len(used)].tolist()))
+    canary = np.uint16(0x7FC1)
+    k2 = np.full((n_dst,) + k.shape[1:], canary, np.uint16)
+    v2 = np.full((n_dst,) + v.shape[1:], canary, np.uint16)
+    src = np.array(used, np.int32)
+    dst = np.array([new_of[p] for p in used], np.int32)
+    k_before, v_before = k.copy(), v.copy()
+    assert oracle.copy_pages(k2, v2, k, v, dst, src) == 0
+    assert np.array_equal(k, k_before) and np.array_equal(v, v_before)
+    assert np.array_equal(k2[dst], k[src]) and np.array_equal(v2[dst], v[src])
+    rest = np.setdiff1d(np.arange(n_dst), dst)
+    assert (k2[rest] == canary).all() and (v2[rest] == canary).all()
+    bt2 = b.block_tables.copy()
+    for s in range(b.batch):
+        for i in range((int(b.ctx_lens[s]) + 15) // 16):
+            bt2[s, i] = new_of[int(b.block_tables[s, i])]
+    o2, l2 = oracle.attention(k2, v2, b.q_lens, b.ctx_lens, bt2, b.q)
+    assert np.array_equal(o2, o_ref) and np.array_equal(l2, l_ref)
+    # inside one pool the copies are simultaneous: a rotation a -> b -> c -> a
+    a, bb, c = used[0], used[1], used[2]
+    kr, vr = k.copy(), v.copy()
+    assert oracle.copy_pages(kr, vr, kr, vr, [bb, c, a], [a, bb, c]) == 0
+    ke, ve = k.copy(), v.copy()
+    ke[[bb, c, a]] = k[[a, bb, c]]
+    ve[[bb, c, a]] = v[[a, bb, c]]
+    assert np.array_equal(kr, ke) and np.array_equal(vr, ve)
+    assert not np.array_equal(k[a], v[a])                       # the planes differ, so a K/V mix-up shows
+    # refusals write nothing
+    for bad_dst, bad_src in (([n_dst], [used[0]]), ([0], [b.num_pages]), ([-1], [used[0]]), ([3, 3], [used[0], used[1]])):
+        k3, v3 = k2.copy(), v2.copy()
+        assert oracle.copy_pages(k3, v3, k, v, bad_dst, bad_src) == -1
+        assert np.array_equal(k3, k2) and np.array_equal(v3, v2)
+    assert oracle.copy_pages(k2, v2, k, v, [], []) == 0
+
+
 PINS = [pin_dense_bruteforce, pin_rows_sum_to_one, pin_single_token_returns_v,
         pin_identical_keys_give_mean_of_v, pin_two_key_closed_form, pin_gqa_head_mapping,
         pin_page_permutation_invariance, pin_split_merge_identity, pin_chunking_identity,
-        pin_append_replay]
+        pin_append_replay, pin_page_copy_migration]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda f: f.__name__)
@@ -264,6 +310,11 @@ MUTATIONS = [
     ("merge weights by exp(lse_k - m*) unnormalised", "double w = exp(lse_parts[k] - *lse);", "double w = exp(lse_parts[k] - mstar);"),
     ("V read from the K plane", "const uint16_t *vj = V + pool_off(bt[j / ORACLE_PAGE], g, j % ORACLE_PAGE, Hkv, d);\n        for (int c = 0; c < d; ++c) out[c] += x[j] * bf16_to_f64(vj[c]);",
      "const uint16_t *vj = K + pool_off(bt[j / ORACLE_PAGE], g, j % ORACLE_PAGE, Hkv, d);\n        for (int c = 0; c < d; ++c) out[c] += x[j] * bf16_to_f64(vj[c]);"),
+    ("page copy takes V from the K plane", "V_src + (size_t)src_ids[i] * page_elems", "K_src + (size_t)src_ids[i] * page_elems"),
+    ("page copy reads the destination's page number", "K_src + (size_t)src_ids[i] * page_elems", "K_src + (size_t)dst_ids[i] * page_elems"),
+    ("page copy forgets the kv heads in the page size", "const size_t page_elems = (size_t)Hkv * ORACLE_PAGE * (size_t)d;",
+     "const size_t page_elems = (size_t)ORACLE_PAGE * (size_t)d;"),
+    ("page copy writes V pages into the K plane", "memcpy(V_dst + (size_t)dst_ids[i] * page_elems", "memcpy(K_dst + (size_t)dst_ids[i] * page_elems"),
     ("bf16 widened from the low half", "uint32_t u = (uint32_t)b << 16;", "uint32_t u = (uint32_t)b << 15;"),
 ]
 
