@@ -314,6 +314,63 @@ def run_trace_bench(args):
     }))
 
 
+def run_page_copy_bench(args):
+    """--page-copy: every used page of config 2 (534 MB of K+V) moves to a second pool in one call,
+    alternating between two destination pools; bytes read + written against the measured copy bandwidth."""
+    import torch
+    import paper_2604_07144_b200 as ap
+    torch.cuda.set_device(0)
+    batch = make_batch(2)
+    hkv, d = batch.num_kv_heads, batch.head_dim
+    used = np.array(sorted({int(batch.block_tables[s, i]) for s in range(batch.batch)
+                            for i in range((int(batch.ctx_lens[s]) + 15) // 16)}), np.int32)
+    to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    src_planes = (to_dev(batch.k_pool), to_dev(batch.v_pool))
+    src = ap.kv_pool_create(batch.num_pages, hkv, d, *src_planes)
+    n_dst = len(used)
+    dsts = []
+    for i in range(3):
+        planes = (torch.zeros((n_dst, hkv, 16, d), dtype=torch.bfloat16, device="cuda"),
+                  torch.zeros((n_dst, hkv, 16, d), dtype=torch.bfloat16, device="cuda"))
+        dsts.append((ap.kv_pool_create(n_dst, hkv, d, *planes), planes,
+                     np.random.default_rng(i).permutation(n_dst).astype(np.int32)))
+    page_bytes = 2 * hkv * 16 * d * 2
+    moved = 2 * len(used) * page_bytes                        # read + written
+    for i in range(max(args.warmup, 3)):
+        ap.kv_copy_pages(dsts[i % 3][0], src, dsts[i % 3][2], used)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        ap.kv_copy_pages(dsts[i % 3][0], src, dsts[i % 3][2], used)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    # device-only time of the kernel: the pair list of every call is already queued behind the previous call
+    peaks = measured_peaks()
+    gbs = moved / (ms * 1e-3) / 1e9
+    assert all(ap.last_device_status(p[0]) == 0 for p in dsts)
+    print(json.dumps({
+        "metric": "kv_page_copy_bytes_per_s", "value": gbs, "unit": "GB/s (read + written)", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": "config2_used_pages_to_a_second_pool", "pages": int(len(used)), "page_bytes": page_bytes,
+                   "l2": "three destination pools in rotation; source 534 MB > 126 MB L2",
+                   "includes": "upload of the page-pair list (65 KB) and the copy kernel"},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "kernel": "kv_copy_pages", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}", "traffic": None,
+                     "bytes_per_launch": moved, "us_per_launch": ms * 1e3},
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
+    }))
+    for p, _, _ in dsts:
+        ap.kv_pool_destroy(p)
+    ap.kv_pool_destroy(src)
+
+
 def main():
     ap_ = argparse.ArgumentParser()
     ap_.add_argument("--gpus", type=int, default=1)
@@ -323,6 +380,8 @@ def main():
     ap_.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
     ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
     ap_.add_argument("--no-cpu-baseline", action="store_true")
+    ap_.add_argument("--page-copy", action="store_true",
+                     help="time ap_kv_copy_pages on config 2's used pages instead of the serving iteration")
     ap_.add_argument("--side-by-side", type=int, default=None,
                      help="mixed iterations: 0 = decode then prefill, 1 = planner decides (library default), "
                           "k >= 2 = decode on k CTAs next to prefill")
@@ -331,6 +390,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args)
+        return
+
+    if args.page_copy:
+        run_page_copy_bench(args)
         return
 
     if args.config == 5:

@@ -197,6 +197,27 @@ int ap_plan_export(const ap_plan *plan, int32_t *blob, size_t capacity_ints, ap_
 /* --------------------------------------------------------------- kernels -- */
 
 /*
+ * KV page copy (Sec. 5.1, execution model, Phase 2 "Reconfiguration": moving
+ * from one serving plan to the next migrates KV caches; the page is the unit
+ * that moves).  For i in [0, n): page src_ids[i] of src_pool -- every kv head,
+ * every slot, K and V -- is copied bit for bit to page dst_ids[i] of dst_pool.
+ * The pools must have the same kv heads, head_dim and page size (else
+ * INVALID_ARG) and live on the same device (else UNSUPPORTED: a move between
+ * GPUs is the caller's peer copy); they may be the same pool (copy-on-write of
+ * a shared prefix page).  dst_ids, src_ids: host, n entries each; they are read
+ * before the call returns.  An id out of range -> BAD_BLOCK_TABLE; a
+ * destination listed twice, or, inside one pool, a destination that is also
+ * another pair's source -> INVALID_ARG (the copies run in parallel); a page
+ * copied onto itself is skipped.  Nothing is queued when an error is
+ * returned.  Neither pool's allocator state changes: allocate the destination
+ * pages and free the source pages with the calls above.  Stream-ordered, no
+ * host synchronisation: a following ap_kv_append / ap_attention_iteration on
+ * the same stream sees the copied pages.  Host-only pools: validation only.
+ */
+int ap_kv_copy_pages(ap_kv_pool *dst_pool, const ap_kv_pool *src_pool, int32_t n, const int32_t *dst_ids,
+                     const int32_t *src_ids, void *stream);
+
+/*
  * KV append (App. B Eq. "serve-latency": every step extends the context).
  * Token t of sequence s sits at position p = ctx_len - q_len + t and is copied,
  * bit for bit, to K/V[block_table[s][p/16]][kv_head][p%16][:].

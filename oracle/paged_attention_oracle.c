@@ -19,7 +19,7 @@
  *              page  = block_table[s][p div 16], slot = p mod 16;
  *              K[page][kv_head][slot][:] <- k_new[row][kv_head][:]  (bit copy)
  *   page copy: page src_ids[i] (all kv heads, K and V) -> page dst_ids[i], all
- *              pairs at once (KV-cache migration between plans, Sec. 3.2)
+ *              pairs at once (KV-cache migration between plans, Sec. 5.1 Phase 2)
  *   attention: query row (s,t), q head h, kv head g = h div (Hq/Hkv):
  *              x_j = scale * <q, k_j>  for j = 0..p   (causal bound j <= p)
  *              m = max_j x_j,  l = sum_j exp(x_j - m)
@@ -99,7 +99,7 @@ int oracle_kv_append(uint16_t *K, uint16_t *V, int num_pages, int Hkv, int d,
 }
 
 /*
- * KV page copy (Sec. 3.2, Phase 2 "Reconfiguration": the transition between two
+ * KV page copy (Sec. 5.1, execution model, Phase 2 "Reconfiguration": the transition between two
  * plans migrates KV caches; a page is the unit that moves).  For i = 0..n-1 the
  * whole page src_ids[i] of the source planes -- every kv head, every slot, both
  * K and V -- is copied bit for bit to page dst_ids[i] of the destination

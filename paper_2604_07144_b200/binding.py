@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "ap_status_string", "ap_kv_pool_bytes", "ap_kv_pool_create", "ap_kv_pool_destroy",
     "ap_kv_pool_k_base", "ap_kv_pool_v_base", "ap_kv_pool_alloc_pages", "ap_kv_pool_free_pages",
     "ap_kv_pool_seed_free_list", "ap_kv_pool_num_free", "ap_kv_pool_set_side_by_side", "ap_plan_create", "ap_plan_destroy",
-    "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append",
+    "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append", "ap_kv_copy_pages",
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
     "ap_static_workspace_bytes", "ap_attention_iteration_static",
@@ -116,6 +116,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_plan_get_info": (ctypes.c_int, [vp, ctypes.POINTER(PlanInfo)]),
         "ap_plan_export": (ctypes.c_int, [vp, vp, sz, ctypes.POINTER(PlanLayout)]),
         "ap_kv_append": (ctypes.c_int, [vp, vp, vp, vp, vp]),
+        "ap_kv_copy_pages": (ctypes.c_int, [vp, vp, i32, vp, vp, vp]),
         "ap_attention_iteration": (ctypes.c_int, [vp, vp, vp, vp, vp, vp, sz, vp]),
         "ap_serving_iteration_host": (ctypes.c_int, [vp, ctypes.POINTER(BatchDesc), vp, vp, vp, vp, vp, vp]),
         "ap_last_device_status": (ctypes.c_int, [vp, vp]),
@@ -311,6 +312,16 @@ def plan_export(plan: Plan) -> dict:
 def kv_append(pool: KVPool, plan: Plan, k_new, v_new, stream=None) -> None:
     _check(load().ap_kv_append(pool.handle, plan.handle, _ptr(k_new), _ptr(v_new), _stream(stream)),
            "ap_kv_append")
+
+
+def kv_copy_pages(dst_pool: KVPool, src_pool: KVPool, dst_ids: Sequence[int], src_ids: Sequence[int], stream=None) -> None:
+    """Page ``src_ids[i]`` of ``src_pool`` -> page ``dst_ids[i]`` of ``dst_pool`` (all kv heads, K and V)."""
+    dst = np.ascontiguousarray(dst_ids, dtype=np.int32)
+    src = np.ascontiguousarray(src_ids, dtype=np.int32)
+    if dst.shape != src.shape or dst.ndim != 1:
+        raise ValueError("dst_ids and src_ids must be 1-D and of the same length")
+    _check(load().ap_kv_copy_pages(dst_pool.handle, src_pool.handle, int(dst.size), dst.ctypes.data, src.ctypes.data,
+                                   _stream(stream) if dst_pool.desc.device >= 0 else None), "ap_kv_copy_pages")
 
 
 def attention_iteration(pool: KVPool, plan: Plan, q, out, lse=None, workspace=None,

@@ -648,6 +648,53 @@ int ap_kv_append(ap_kv_pool *pool, const ap_plan *plan, const void *k_new, const
     return AP_OK;
 }
 
+int ap_kv_copy_pages(ap_kv_pool *dst_pool, const ap_kv_pool *src_pool, int32_t n, const int32_t *dst_ids,
+                     const int32_t *src_ids, void *stream) {
+    if (!dst_pool || !src_pool || n < 0 || (n > 0 && (!dst_ids || !src_ids))) return AP_ERR_INVALID_ARG;
+    const ap_pool_desc &dd = dst_pool->desc, &sd = src_pool->desc;
+    if (dd.num_kv_heads != sd.num_kv_heads || dd.head_dim != sd.head_dim || dd.page_size != sd.page_size)
+        return AP_ERR_INVALID_ARG;
+    if ((dd.device < 0) != (sd.device < 0) || (dd.device >= 0 && dd.device != sd.device)) return AP_ERR_UNSUPPORTED;
+    // Validation on the host, before anything is queued.  The copies run in parallel, so a
+    // destination may appear once only and, inside one pool, may not be another pair's source.
+    const bool same = dst_pool == src_pool || (dd.device >= 0 && dd.k_base == sd.k_base);
+    std::vector<uint8_t> is_dst((size_t)dd.num_pages, 0);
+    std::vector<int32_t> pairs;
+    pairs.reserve(2 * (size_t)n);
+    for (int32_t i = 0; i < n; ++i) {
+        if (dst_ids[i] < 0 || dst_ids[i] >= dd.num_pages || src_ids[i] < 0 || src_ids[i] >= sd.num_pages)
+            return AP_ERR_BAD_BLOCK_TABLE;
+        if (is_dst[(size_t)dst_ids[i]]) return AP_ERR_INVALID_ARG;
+        is_dst[(size_t)dst_ids[i]] = 1;
+        if (same && dst_ids[i] == src_ids[i]) continue;           // a page copied onto itself: nothing to do
+        pairs.push_back(dst_ids[i]);
+        pairs.push_back(src_ids[i]);
+    }
+    if (same)
+        for (int32_t i = 0; i < n; ++i)
+            if (dst_ids[i] != src_ids[i] && is_dst[(size_t)src_ids[i]]) return AP_ERR_INVALID_ARG;
+    if (pairs.empty() || dd.device < 0) return AP_OK;             // a host-only pool has no planes to copy
+    DeviceGuard guard(dd.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    PlanBuffer buf;
+    int rc = acquire_plan_buffer(dst_pool, pairs.size(), &buf);
+    if (rc != AP_OK) return rc;
+    std::memcpy(buf.host, pairs.data(), pairs.size() * sizeof(int32_t));
+    cudaError_t e = cudaMemcpyAsync(buf.dev, buf.host, pairs.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = launch_kv_copy_pages(dst_pool, src_pool, buf.dev, (int)(pairs.size() / 2), st);
+    // the staging area is free again once the kernel has read the pair list
+    if (e == cudaSuccess) e = cudaEventRecord(buf.uploaded, st);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        (void)cudaStreamSynchronize(st);
+        release_plan_buffer(buf);
+        return AP_ERR_CUDA;
+    }
+    dst_pool->plan_buffers.push_back(buf);
+    return AP_OK;
+}
+
 int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
                            void *workspace, size_t workspace_bytes, void *stream) {
     if (!pool || !plan || plan->pool != pool) return AP_ERR_INVALID_ARG;

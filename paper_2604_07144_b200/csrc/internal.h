@@ -133,6 +133,9 @@ cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, co
                                  float *lse, float *o_part, float *lse_part, cudaStream_t stream);
 cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                            float *lse, cudaStream_t stream);
+// d_pairs: device [n_pairs][2] = (destination page, source page)
+cudaError_t launch_kv_copy_pages(const ap_kv_pool *dst_pool, const ap_kv_pool *src_pool, const int32_t *d_pairs,
+                                 int n_pairs, cudaStream_t stream);
 
 // Launch with programmatic stream serialization: the kernel may begin (up to its griddep_wait)
 // before the previous kernel in the stream has drained, which hides launch latency and preamble.

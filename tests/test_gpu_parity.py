@@ -132,6 +132,90 @@ def test_iteration_is_capturable_in_a_cuda_graph(mode):
         run.close()
 
 
+def _used_pages(batch):
+    return sorted({int(batch.block_tables[s, i]) for s in range(batch.batch)
+                   for i in range((int(batch.ctx_lens[s]) + 15) // 16)})
+
+
+@pytest.mark.parametrize("shape", [W.SHAPE_8B, (8, 2, 64)], ids=["8B", "S1"])
+def test_page_copy_migration_and_copy_on_write(shape):
+    """ap_kv_copy_pages against the oracle, bit for bit: every used page of a batch moves to a second
+    pool (canaries elsewhere stay, the source is untouched), attention through the remapped block
+    tables still matches the oracle; then pages are duplicated inside one pool."""
+    import torch
+    import oracle
+    from harness import compare_outputs, to_dev
+    batch = W._assemble("migrate", shape, W.make_rng(51), np.array([1, 70, 1, 1, 3], np.int32),
+                        np.array([300, 200, 17, 1025, 64], np.int32), 1.3)
+    run = GpuRun(batch)
+    try:
+        run.append()
+        used = _used_pages(batch)
+        rng = np.random.default_rng(3)
+        n_dst = batch.num_pages + 9
+        new_of = dict(zip(used, rng.permutation(n_dst)[:len(used)].tolist()))
+        src = np.array(used, np.int32)
+        dst = np.array([new_of[p] for p in used], np.int32)
+        canary = np.full((n_dst,) + batch.k_pool.shape[1:], 0x7FC1, np.uint16)
+        k2, v2 = to_dev(canary), to_dev(canary)
+        pool2 = ap.kv_pool_create(n_dst, batch.num_kv_heads, batch.head_dim, k2, v2)
+        ap.kv_copy_pages(pool2, run.pool, dst, src)
+        # the oracle's version of the same move
+        k_src, v_src = to_bits(run.k_pool), to_bits(run.v_pool)
+        k_ref, v_ref = canary.copy(), canary.copy()
+        assert oracle.copy_pages(k_ref, v_ref, k_src, v_src, dst, src) == 0
+        assert ap.last_device_status(pool2) == 0
+        assert np.array_equal(to_bits(k2), k_ref) and np.array_equal(to_bits(v2), v_ref)
+        assert np.array_equal(to_bits(run.k_pool), k_src) and np.array_equal(to_bits(run.v_pool), v_src)
+        # attention on the migrated pages (no new tokens are appended again: same contexts, remapped tables)
+        bt2 = batch.block_tables.copy()
+        for s in range(batch.batch):
+            for i in range((int(batch.ctx_lens[s]) + 15) // 16):
+                bt2[s, i] = new_of[int(batch.block_tables[s, i])]
+        plan2 = ap.plan_create(pool2, batch.q_lens, batch.ctx_lens, bt2, batch.num_q_heads)
+        ws = torch.empty(max(ap.plan_workspace_bytes(plan2), 256), dtype=torch.uint8, device="cuda:0")
+        ap.attention_iteration(pool2, plan2, run.q, run.out, run.lse, ws, ap.plan_workspace_bytes(plan2))
+        assert ap.last_device_status(pool2) == 0
+        ref_out, ref_lse = oracle.attention(k_ref, v_ref, batch.q_lens, batch.ctx_lens, bt2, batch.q)
+        compare_outputs(to_bits(run.out)[:batch.n_new], run.lse.cpu().numpy()[:batch.n_new], ref_out, ref_lse, "migrated")
+        ap.plan_destroy(plan2)
+        # copy-on-write inside the second pool: duplicate some pages into free ones
+        free = np.setdiff1d(np.arange(n_dst), dst).astype(np.int32)[:5]
+        cow_src = dst[:len(free)]
+        ap.kv_copy_pages(pool2, pool2, free, cow_src)
+        assert oracle.copy_pages(k_ref, v_ref, k_ref, v_ref, free, cow_src) == 0
+        assert np.array_equal(to_bits(k2), k_ref) and np.array_equal(to_bits(v2), v_ref)
+        # a refused call queues nothing
+        with pytest.raises(ap.ApError):
+            ap.kv_copy_pages(pool2, pool2, [int(free[0]), int(free[1])], [int(cow_src[0]), int(free[0])])
+        assert np.array_equal(to_bits(k2), k_ref)
+        ap.kv_pool_destroy(pool2)
+    finally:
+        run.close()
+
+
+def test_page_copy_full_size_config2():
+    """All 8 k used pages of config 2 (534 MB) in one call, compared bit for bit with the oracle."""
+    import oracle
+    from harness import to_dev
+    batch = W.config2()
+    used = np.array(_used_pages(batch), np.int32)
+    k1, v1 = to_dev(batch.k_pool), to_dev(batch.v_pool)
+    pool1 = ap.kv_pool_create(batch.num_pages, batch.num_kv_heads, batch.head_dim, k1, v1)
+    n_dst = len(used) + 3
+    dst = np.random.default_rng(5).permutation(n_dst)[:len(used)].astype(np.int32)
+    canary = np.full((n_dst,) + batch.k_pool.shape[1:], 0x7FC1, np.uint16)
+    k2, v2 = to_dev(canary), to_dev(canary)
+    pool2 = ap.kv_pool_create(n_dst, batch.num_kv_heads, batch.head_dim, k2, v2)
+    ap.kv_copy_pages(pool2, pool1, dst, used)
+    assert ap.last_device_status(pool2) == 0
+    k_ref, v_ref = canary.copy(), canary.copy()
+    assert oracle.copy_pages(k_ref, v_ref, batch.k_pool, batch.v_pool, dst, used) == 0
+    assert np.array_equal(to_bits(k2), k_ref) and np.array_equal(to_bits(v2), v_ref)
+    ap.kv_pool_destroy(pool1)
+    ap.kv_pool_destroy(pool2)
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]

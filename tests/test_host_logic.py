@@ -213,6 +213,31 @@ def test_side_by_side_planning():
     ap.kv_pool_destroy(pool)
 
 
+def test_copy_pages_validation_on_host_pools():
+    """ap_kv_copy_pages checks its lists on the host before anything is queued."""
+    a, b = host_pool(20), host_pool(30)
+    ap.kv_copy_pages(b, a, [], [])
+    ap.kv_copy_pages(b, a, [29, 0, 7], [19, 19, 3])            # one source to several destinations is fine
+    ap.kv_copy_pages(a, a, [5, 6], [5, 1])                     # a page onto itself is skipped
+    for dst, src, status in (([30], [0], B.AP_ERR_BAD_BLOCK_TABLE), ([0], [20], B.AP_ERR_BAD_BLOCK_TABLE),
+                             ([-1], [0], B.AP_ERR_BAD_BLOCK_TABLE), ([4, 4], [1, 2], B.AP_ERR_INVALID_ARG)):
+        with pytest.raises(ap.ApError) as e:
+            ap.kv_copy_pages(b, a, dst, src)
+        assert e.value.status == status
+    # inside one pool a destination may not be another pair's source (the copies run in parallel)
+    with pytest.raises(ap.ApError) as e:
+        ap.kv_copy_pages(a, a, [1, 2], [0, 1])
+    assert e.value.status == B.AP_ERR_INVALID_ARG
+    other_shape = ap.kv_pool_create(20, 4, 64, device=-1)
+    with pytest.raises(ap.ApError) as e:
+        ap.kv_copy_pages(other_shape, a, [0], [0])
+    assert e.value.status == B.AP_ERR_INVALID_ARG
+    with pytest.raises(ValueError):
+        ap.kv_copy_pages(b, a, [1, 2], [1])
+    for p in (a, b, other_shape):
+        ap.kv_pool_destroy(p)
+
+
 def test_empty_batch_plans_to_nothing():
     pool = host_pool()
     p = ap.plan_create(pool, [], [], np.zeros((0, 1), np.int32), 8)
