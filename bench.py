@@ -584,6 +584,10 @@ def main():
                                "prefill": paper_model_us(alg["prefill_flops"], alg["prefill_kernel"], peaks),
                                "note": "T_op = F / min(F/A * B, F_peak) with this GPU's measured copy bandwidth and "
                                        "bf16 peak; compare with kernels.*.us_per_launch"},
+            "prediction": {**{k: v for k, v in ap.plan_predict(plans[0], peaks["hbm_gbs"], peaks["bf16_tflops"]).items()
+                              if k.endswith("_us")},
+                           "note": "ap_plan_predict: roofline_* = the paper's operator model computed by the library, "
+                                   "model_* = the planner's calibrated cost model; compare model_step_us with ms_per_step"},
             "prefill_tflops": (alg["prefill_flops"] / (kernels["prefill"]["us_per_launch"] * 1e-6) / 1e12
                                if kernels.get("prefill", {}).get("us_per_launch") else None),
             "step_gbs": alg["total"] / (ms_per_step * 1e-3) / 1e9,

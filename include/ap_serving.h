@@ -177,6 +177,29 @@ typedef struct ap_plan_info {
 int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
 
 /*
+ * Predicted time of a plan's kernels (App. B, "Roofline-Based Serve Cost").
+ * *_bytes / *_flops: the algorithmic work of one attention layer -- every
+ * attended KV token's K and V once per kv head, q read, out and lse written,
+ * used block-table entries once, new K/V read and written once; 4 * head_dim
+ * flop per (q head, query row, unmasked key).
+ * roofline_*_us: the paper's operator model, Eq. "roofline":
+ *   pi = min(F / A * B_g, F_g),  T_op = F / pi   (an operator without flops: A / B_g)
+ * with B_g = hbm_gbs (GB/s) and F_g = tensor_tflops (TFLOP/s); a value <= 0
+ * selects the figures measured on B200 (6448 GB/s copy bandwidth, 1642 TFLOP/s
+ * dense bf16).
+ * model_*_us: the cost model the planner itself uses, calibrated on B200 (per-SM
+ * decode bandwidth, per-step and per-unit prefill cost, fixed costs);
+ * model_step_us accounts for decode running beside prefill when the plan does.
+ * Pure host arithmetic on the plan; works on host-only pools.
+ */
+typedef struct ap_plan_prediction {
+    double decode_bytes, decode_flops, prefill_bytes, prefill_flops, append_bytes;
+    double roofline_decode_us, roofline_prefill_us, roofline_append_us;
+    double model_decode_us, model_prefill_us, model_step_us;
+} ap_plan_prediction;
+int ap_plan_predict(const ap_plan *plan, double hbm_gbs, double tensor_tflops, ap_plan_prediction *out);
+
+/*
  * Host copy of the work lists a plan uploads, for inspection and tests.  The
  * blob is an int32 array; the layout gives the offset (in int32 units) of each
  * section:

@@ -35,7 +35,7 @@ EXPORTED_SYMBOLS = (
     "ap_status_string", "ap_kv_pool_bytes", "ap_kv_pool_create", "ap_kv_pool_destroy",
     "ap_kv_pool_k_base", "ap_kv_pool_v_base", "ap_kv_pool_alloc_pages", "ap_kv_pool_free_pages",
     "ap_kv_pool_seed_free_list", "ap_kv_pool_num_free", "ap_kv_pool_set_side_by_side", "ap_plan_create", "ap_plan_destroy",
-    "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_export", "ap_kv_append", "ap_kv_copy_pages",
+    "ap_plan_workspace_bytes", "ap_plan_get_info", "ap_plan_predict", "ap_plan_export", "ap_kv_append", "ap_kv_copy_pages",
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
     "ap_static_workspace_bytes", "ap_attention_iteration_static",
@@ -69,6 +69,16 @@ class PlanInfo(ctypes.Structure):
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+
+class PlanPrediction(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in (
+        "decode_bytes", "decode_flops", "prefill_bytes", "prefill_flops", "append_bytes",
+        "roofline_decode_us", "roofline_prefill_us", "roofline_append_us",
+        "model_decode_us", "model_prefill_us", "model_step_us")]
+
+    def as_dict(self):
+        return {n: float(getattr(self, n)) for n, _ in self._fields_}
 
 
 class PlanLayout(ctypes.Structure):
@@ -113,6 +123,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_plan_create": (ctypes.c_int, [ctypes.POINTER(vp), vp, ctypes.POINTER(BatchDesc), vp]),
         "ap_plan_destroy": (ctypes.c_int, [vp]),
         "ap_plan_workspace_bytes": (sz, [vp]),
+        "ap_plan_predict": (ctypes.c_int, [vp, ctypes.c_double, ctypes.c_double, ctypes.POINTER(PlanPrediction)]),
         "ap_plan_get_info": (ctypes.c_int, [vp, ctypes.POINTER(PlanInfo)]),
         "ap_plan_export": (ctypes.c_int, [vp, vp, sz, ctypes.POINTER(PlanLayout)]),
         "ap_kv_append": (ctypes.c_int, [vp, vp, vp, vp, vp]),
@@ -283,6 +294,14 @@ def plan_get_info(plan: Plan) -> dict:
     info = PlanInfo()
     _check(load().ap_plan_get_info(plan.handle, ctypes.byref(info)), "ap_plan_get_info")
     return info.as_dict()
+
+
+def plan_predict(plan: Plan, hbm_gbs: float = 0.0, tensor_tflops: float = 0.0) -> dict:
+    """Algorithmic work and predicted kernel times of a plan (paper's roofline model and the planner's own)."""
+    est = PlanPrediction()
+    _check(load().ap_plan_predict(plan.handle, float(hbm_gbs), float(tensor_tflops), ctypes.byref(est)),
+           "ap_plan_predict")
+    return est.as_dict()
 
 
 def plan_export(plan: Plan) -> dict:

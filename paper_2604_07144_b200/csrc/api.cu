@@ -97,6 +97,10 @@ constexpr double kDecodeGpuGBs = 6000.0;     // GB/s decode reaches with all SMs
 constexpr double kPrefillStepUs = 2.1;       // one 128-key step of a two-tile unit at d = 128
 constexpr double kPrefillStepSingleUs = 1.5; // the same for a one-tile unit
 constexpr double kPrefillUnitUs = 5.3;       // prologue + epilogue + relaunch gap of a unit
+constexpr double kPrefillTailUs = 12.0;      // spread of the SMs' finishing times (about half a short unit) + ramp-up
+constexpr double kDecodeFixedUs = 8.0;       // first-data latency and finishing spread of the decode kernel
+constexpr double kAppendGBs = 4000.0;        // scatter of 256-byte rows
+constexpr double kAppendFixedUs = 3.0;
 
 int side_by_side_decode_ctas(const ap_kv_pool *pool, const ap_batch_desc *b, int d, int Hkv, int G, int max_ctas) {
     const int mode = pool->side_by_side_mode;
@@ -348,6 +352,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     // ---- validation + row bookkeeping
     int64_t n_new = 0, kv_tokens = 0, bt_total = 0, pairs = 0;
     int64_t decode_rows = 0, prefill_seqs = 0;
+    int64_t decode_kv = 0, decode_bt = 0, prefill_kv = 0, prefill_rows = 0;   // for the work figures of ap_plan_predict
     for (int s = 0; s < B; ++s) {
         const int32_t ql = b->q_lens[s], cl = b->ctx_lens[s];
         if (ql < 0 || cl < 0 || ql > cl) return AP_ERR_INVALID_ARG;
@@ -362,6 +367,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
         bt_total += need;
         if (ql == 1) ++decode_rows; else ++prefill_seqs;
         if (ql > 1) pairs += (int64_t)ql * (cl - ql) + (int64_t)ql * (ql + 1) / 2;
+        if (ql == 1) { decode_kv += cl; decode_bt += need; } else { prefill_kv += cl; prefill_rows += ql; }
     }
     if (n_new > (int64_t)1 << 30) return AP_ERR_UNSUPPORTED;
 
@@ -600,9 +606,61 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     info.prefill_tiles = (int64_t)tiles.size();
     info.launches_append = n_new > 0 ? 1 : 0;
     info.launches_attention = (items.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
+    {
+        // algorithmic work of one layer: every attended KV token's K and V once per kv head, q read,
+        // out + lse written, used block-table entries once; 4 d flop per (q head, query row, unmasked key)
+        const double per_kv_token = 2.0 * (double)Hkv * (double)d * 2.0;
+        const double per_row = 2.0 * (double)b->num_q_heads * (double)d * 2.0 + (double)b->num_q_heads * 4.0;
+        plan->work.decode_bytes = (double)decode_kv * per_kv_token + (double)decode_rows * per_row + (double)decode_bt * 4.0;
+        plan->work.prefill_bytes = (double)prefill_kv * per_kv_token + (double)prefill_rows * per_row;
+        plan->work.append_bytes = 2.0 * (double)n_new * per_kv_token;
+        plan->work.decode_flops = 4.0 * (double)b->num_q_heads * (double)d * (double)decode_kv;
+        plan->work.prefill_flops = 4.0 * (double)b->num_q_heads * (double)d * (double)pairs;
+        double w_p = 0.0;
+        for (const PrefillTile &t : tiles) {
+            const int steps = (t.pos0 + t.rows + 127) / 128;
+            w_p += steps * (t.q_head_b >= 0 ? kPrefillStepUs : kPrefillStepSingleUs) * ((double)d / 128.0) + kPrefillUnitUs;
+        }
+        plan->work.prefill_sm_us = w_p;
+    }
     plan->side_by_side = side_ctas > 0 && !items.empty() && !tiles.empty();
     info.side_by_side = plan->side_by_side ? 1 : 0;
     *out = plan;
+    return AP_OK;
+}
+
+int ap_plan_predict(const ap_plan *plan, double hbm_gbs, double tensor_tflops, ap_plan_prediction *out) {
+    if (!plan || !out || !plan->pool) return AP_ERR_INVALID_ARG;
+    const double B = (hbm_gbs > 0.0 ? hbm_gbs : 6448.0) * 1e9;             // bytes / s
+    const double F = (tensor_tflops > 0.0 ? tensor_tflops : 1642.0) * 1e12; // flop / s
+    const PlanWork &w = plan->work;
+    ap_plan_prediction e{};
+    e.decode_bytes = w.decode_bytes;
+    e.decode_flops = w.decode_flops;
+    e.prefill_bytes = w.prefill_bytes;
+    e.prefill_flops = w.prefill_flops;
+    e.append_bytes = w.append_bytes;
+    // Eq. "roofline": pi = min(F/A * B_g, F_g), T_op = F / pi; an operator without flops moves its bytes
+    auto t_op_us = [&](double flops, double bytes) {
+        if (bytes <= 0.0) return 0.0;
+        if (flops <= 0.0) return bytes / B * 1e6;
+        return flops / std::min(flops / bytes * B, F) * 1e6;
+    };
+    e.roofline_decode_us = t_op_us(w.decode_flops, w.decode_bytes);
+    e.roofline_prefill_us = t_op_us(w.prefill_flops, w.prefill_bytes);
+    e.roofline_append_us = t_op_us(0.0, w.append_bytes);
+    // calibrated model (the one the planner's side-by-side decision uses)
+    const int sms = plan->pool->sm_count;
+    const double ctas = (double)std::max<int64_t>(plan->info.decode_ctas, 1);
+    const double decode_rate = std::min(ctas * kDecodeSmGBs, kDecodeGpuGBs) * 1e3;        // bytes / us
+    e.model_decode_us = w.decode_bytes > 0.0 ? w.decode_bytes / decode_rate + kDecodeFixedUs : 0.0;
+    e.model_prefill_us = w.prefill_sm_us > 0.0 ? w.prefill_sm_us / sms + kPrefillTailUs : 0.0;
+    const double append_us = w.append_bytes > 0.0 ? w.append_bytes / (kAppendGBs * 1e3) + kAppendFixedUs : 0.0;
+    if (plan->side_by_side)
+        e.model_step_us = append_us + (w.decode_bytes / (kDecodeSmGBs * 1e3) + w.prefill_sm_us) / sms + kPrefillTailUs;
+    else
+        e.model_step_us = append_us + e.model_decode_us + e.model_prefill_us;
+    *out = e;
     return AP_OK;
 }
 

@@ -71,6 +71,11 @@ struct PlanBuffer {            // reusable staging for one plan upload
     cudaEvent_t uploaded = nullptr;
 };
 
+struct PlanWork {              // algorithmic work of a plan (one attention layer), for ap_plan_predict
+    double decode_bytes = 0, decode_flops = 0, prefill_bytes = 0, prefill_flops = 0, append_bytes = 0;
+    double prefill_sm_us = 0;  // SM-time of the prefill units by the planner's cost model
+};
+
 struct TimedLaunch {
     int kernel;
     cudaEvent_t start, stop;
@@ -113,6 +118,7 @@ struct ap_plan {
     ap_plan_layout layout{};
     std::vector<int32_t> blob;   // host copy of the uploaded work lists
     int n_part_slots = 0;
+    ap::PlanWork work{};
     bool side_by_side = false;   // decode on the caller's stream and prefill on the pool's second stream, concurrently
     ap::WorkspaceLayout ws{};
     // device pointers into buf.dev

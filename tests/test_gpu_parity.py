@@ -216,6 +216,35 @@ def test_page_copy_full_size_config2():
     ap.kv_pool_destroy(pool2)
 
 
+@pytest.mark.parametrize("config", [2, 3, 4])
+def test_plan_predict_tracks_the_measured_step(config):
+    """The planner's calibrated model (ap_plan_predict.model_step_us) stays within a factor of the
+    measured device time of append + attention on the full-size workloads, and the paper's roofline
+    time is a lower bound of the measured attention time."""
+    import torch
+    batch = {2: W.config2, 3: W.config3, 4: W.config4}[config]()
+    run = GpuRun(batch)
+    try:
+        pred = ap.plan_predict(run.plan)
+        for _ in range(3):
+            run.append(); run.attend()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 10
+        e0.record()
+        for _ in range(n):
+            run.append(); run.attend()
+        e1.record()
+        torch.cuda.synchronize()
+        assert run.status() == 0
+        us = 1e3 * e0.elapsed_time(e1) / n
+        assert 0.6 * us <= pred["model_step_us"] <= 1.6 * us, (us, pred)
+        # the pool stays in L2 only for small workloads; these are all larger than L2
+        assert max(pred["roofline_decode_us"], pred["roofline_prefill_us"]) <= 1.1 * us
+    finally:
+        run.close()
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]

@@ -238,6 +238,43 @@ def test_copy_pages_validation_on_host_pools():
         ap.kv_pool_destroy(p)
 
 
+def test_plan_predict_matches_the_cost_model_oracle():
+    """ap_plan_predict: work figures equal the oracle's counts exactly, the paper-model times to rounding;
+    the planner's own model is positive, additive when sequential and shorter when side by side."""
+    from oracle import roofline_model as R
+    batches = [W.config1(), W.config2(with_pool=False), W.config3(with_pool=False), W.config4(with_pool=False),
+               W.random_ragged(5, batch=6, max_ctx=900, max_q=300), W.random_ragged(21, batch=9, max_ctx=700, max_q=3)]
+    for b in batches:
+        pool = ap.kv_pool_create(b.num_pages, b.num_kv_heads, b.head_dim, device=-1)
+        plan = ap.plan_create(pool, b.q_lens, b.ctx_lens, b.block_tables, b.num_q_heads)
+        for bw, tf in ((0.0, 0.0), (3350.0, 989.0)):
+            got = ap.plan_predict(plan, bw, tf)
+            work = R.iteration_work(b.q_lens, b.ctx_lens, b.num_q_heads, b.num_kv_heads, b.head_dim)
+            for k, v in work.items():
+                assert got[k] == v, (b.name, k)
+            ref = R.iteration_times_us(work, bw or 6448.0, tf or 1642.0)
+            for k, v in ref.items():
+                assert np.isclose(got[k], v, rtol=1e-12, atol=0.0), (b.name, k)
+        info = ap.plan_get_info(plan)
+        assert (got["model_decode_us"] > 0) == (info["decode_rows"] > 0)
+        assert (got["model_prefill_us"] > 0) == (info["prefill_seqs"] > 0)
+        if not info["side_by_side"]:
+            assert got["model_step_us"] >= got["model_decode_us"] + got["model_prefill_us"]
+        ap.plan_destroy(plan)
+        ap.kv_pool_destroy(pool)
+    # config 3: side by side is predicted (and planned) to be shorter than decode then prefill
+    b = W.config3(with_pool=False)
+    steps = {}
+    for mode in (0, 1):
+        pool = ap.kv_pool_create(b.num_pages, b.num_kv_heads, b.head_dim, device=-1)
+        ap.kv_pool_set_side_by_side(pool, mode)
+        plan = ap.plan_create(pool, b.q_lens, b.ctx_lens, b.block_tables, b.num_q_heads)
+        steps[mode] = ap.plan_predict(plan)["model_step_us"]
+        ap.plan_destroy(plan)
+        ap.kv_pool_destroy(pool)
+    assert steps[1] < 0.95 * steps[0]
+
+
 def test_empty_batch_plans_to_nothing():
     pool = host_pool()
     p = ap.plan_create(pool, [], [], np.zeros((0, 1), np.int32), 8)

@@ -263,6 +263,41 @@ def pin_page_copy_migration():
     assert oracle.copy_pages(k2, v2, k, v, [], []) == 0
 
 
+def test_roofline_model_pins():
+    """The cost-model oracle (App. B Eq. "roofline") against what the mathematics fixes."""
+    from oracle import roofline_model as R
+    B, F = 6.0e12, 1.5e15
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        fl, by = float(10 ** rng.uniform(3, 15)), float(10 ** rng.uniform(3, 12))
+        # min over rates = max over times
+        assert np.isclose(R.t_op(fl, by, B, F), max(fl / F, by / B), rtol=1e-12)
+    ridge = F / B                                   # AI* = F_g / B_g: both branches meet
+    assert np.isclose(R.t_op(ridge * 1e9, 1e9, B, F), 1e9 / B, rtol=1e-12)
+    assert np.isclose(R.achieved_rate(ridge * 1e9, 1e9, B, F), F, rtol=1e-12)
+    assert R.t_op(2.0 * ridge * 1e9, 1e9, B, F) == 2.0 * ridge * 1e9 / F          # compute-bound above the ridge
+    assert R.t_op(0.5 * ridge * 1e9, 1e9, B, F) == 1e9 / B                        # memory-bound below it
+    assert R.t_op(0.0, 1e9, B, F) == 1e9 / B and R.t_op(0.0, 0.0, B, F) == 0.0
+    # long-context grouped-query decode: intensity tends to G = Hq / Hkv flop per byte
+    for hq, hkv, d in ((32, 8, 128), (64, 8, 128), (8, 2, 64)):
+        w = R.iteration_work([1], [1 << 20], hq, hkv, d)
+        assert abs(w["decode_flops"] / w["decode_bytes"] - hq / hkv) < 1e-2
+    # a causal chunk: the pair count against an explicit enumeration of (row, key) with key <= position
+    ql, cl, hq, hkv, d = 37, 100, 4, 2, 64
+    pairs = sum(1 for t in range(ql) for j in range(cl) if j <= cl - ql + t)
+    w = R.iteration_work([ql], [cl], hq, hkv, d)
+    assert w["prefill_flops"] == 4 * hq * d * pairs and pairs == ql * (cl - ql) + ql * (ql + 1) // 2
+    assert w["append_bytes"] == 2 * ql * (2 * hkv * d * 2)
+    assert w["prefill_bytes"] == cl * 2 * hkv * d * 2 + ql * (2 * hq * d * 2 + hq * 4)
+    # config 2 at the 8B shape is on the memory side of the ridge, config 3's prefill on the compute side
+    b2 = W.config2(with_pool=False)
+    w2 = R.iteration_work(b2.q_lens, b2.ctx_lens, 32, 8, 128)
+    assert w2["decode_flops"] / w2["decode_bytes"] < 5 < ridge
+    b3 = W.config3(with_pool=False)
+    w3 = R.iteration_work(b3.q_lens, b3.ctx_lens, 32, 8, 128)
+    assert w3["prefill_flops"] / w3["prefill_bytes"] > ridge
+
+
 PINS = [pin_dense_bruteforce, pin_rows_sum_to_one, pin_single_token_returns_v,
         pin_identical_keys_give_mean_of_v, pin_two_key_closed_form, pin_gqa_head_mapping,
         pin_page_permutation_invariance, pin_split_merge_identity, pin_chunking_identity,
