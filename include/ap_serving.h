@@ -15,7 +15,7 @@
  * "serve-latency"); attention heads A_z, KV heads K_z <= A_z, head dimension
  * d_z (App. B, model description); the KV cache is a finite pool counted in
  * tokens (App. B Eq. "oom", theta = 0.8; App. C.2 "token-capacity limits");
- * KV caches are relocatable (Sec. 4.1, Phase 2), hence block-table
+ * KV caches are relocatable (Sec. 5.1, Phase 2), hence block-table
  * indirection; paged KV memory and chunked prefill are the data-plane
  * techniques of the served systems (App. H).  The arithmetic itself is the
  * textbook definition:
@@ -117,7 +117,7 @@ void *ap_kv_pool_v_base(const ap_kv_pool *pool);
 int ap_kv_pool_set_side_by_side(ap_kv_pool *pool, int32_t mode);
 
 /* Host page allocator (per-request page ownership; pages are relocatable units,
- * Sec. 4.1 Phase 2).  alloc is all-or-nothing: OUT_OF_PAGES leaves the free
+ * Sec. 5.1 Phase 2).  alloc is all-or-nothing: OUT_OF_PAGES leaves the free
  * list unchanged.  out_ids / ids: host.  free of a page that is not allocated,
  * out of range or repeated in the call -> INVALID_ARG, nothing freed. */
 int ap_kv_pool_alloc_pages(ap_kv_pool *pool, int32_t n, int32_t *out_ids);

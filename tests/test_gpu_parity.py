@@ -240,7 +240,7 @@ def test_plan_predict_tracks_the_measured_step(config):
         us = 1e3 * e0.elapsed_time(e1) / n
         assert 0.6 * us <= pred["model_step_us"] <= 1.6 * us, (us, pred)
         # the pool stays in L2 only for small workloads; these are all larger than L2
-        assert max(pred["roofline_decode_us"], pred["roofline_prefill_us"]) <= 1.1 * us
+        assert max(pred["roofline_decode_us"], pred["roofline_prefill_us"]) <= 1.2 * us
     finally:
         run.close()
 
