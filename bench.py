@@ -314,6 +314,40 @@ def run_trace_bench(args):
     }))
 
 
+def run_policy_comparison(args):
+    """--config 5 --policies: the workload-shift trace under fixed FCFS policies that differ in token
+    budget and prefill chunk size.  Each replay is scored by Eq. "ttotal" of the paper's execution model
+    with the measured device time of its iterations as the serving cost (a fixed policy never
+    reschedules: one interval, no stale or reconfiguration cost)."""
+    import torch
+    from paper_2604_07144_b200 import execution_model as M
+    from paper_2604_07144_b200.trace_runner import TraceRun
+    torch.cuda.set_device(0)
+    rows = []
+    for budget, chunk in ((8192, 512), (8192, 256), (8192, 1024), (4096, 512), (2048, 256)):
+        per_iter, toks, new = [], 0, 0
+        for replay in range(2):                                  # first replay warms up
+            run = TraceRun(iterations=200, token_budget=budget, chunk=chunk)
+            for st in run.steps():
+                if replay == 1 and st.kv_tokens:
+                    per_iter.append(st.gpu_ms * 1e-3)
+                    toks += st.kv_tokens
+                    new += int(st.q_lens.sum())
+            run.close()
+        fb = M.artifact_feedback(M.intervals_from_iterations(per_iter))
+        rows.append({"token_budget": budget, "chunk": chunk, "iterations": len(per_iter), "new_tokens": new,
+                     "kv_tokens": toks, "T_total_s": fb["T_total"], "N": fb["N"],
+                     "kv_tokens_per_s": toks / fb["T_total"], "new_tokens_per_s": new / fb["T_total"],
+                     "worst_iteration_ms": 1e3 * max(per_iter)})
+    best = min(rows, key=lambda r: r["T_total_s"] / max(r["new_tokens"], 1))
+    print(json.dumps({"metric": "trace_completion_time_per_policy", "unit": "s", "n_gpus": 1, "data": "synthetic",
+                      "config": {"workload": "config5_workload_shift_trace_8b", "iterations": 200,
+                                 "score": "Eq. ttotal with measured append + attention device time of one layer as t_serve; "
+                                          "policies that leave prompts unfinished at iteration 200 serve fewer new tokens, "
+                                          "so compare T_total per new token"},
+                      "policies": rows, "best_per_new_token": {k: best[k] for k in ("token_budget", "chunk")}}))
+
+
 def run_page_copy_bench(args):
     """--page-copy: every used page of config 2 (534 MB of K+V) moves to a second pool in one call,
     alternating between two destination pools; bytes read + written against the measured copy bandwidth."""
@@ -380,6 +414,9 @@ def main():
     ap_.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
     ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
     ap_.add_argument("--no-cpu-baseline", action="store_true")
+    ap_.add_argument("--policies", action="store_true",
+                     help="with --config 5: replay the trace under several fixed scheduling policies (token budget, "
+                          "prefill chunk) and score each by the paper's trace completion time on measured iterations")
     ap_.add_argument("--page-copy", action="store_true",
                      help="time ap_kv_copy_pages on config 2's used pages instead of the serving iteration")
     ap_.add_argument("--side-by-side", type=int, default=None,
@@ -394,6 +431,10 @@ def main():
 
     if args.page_copy:
         run_page_copy_bench(args)
+        return
+
+    if args.config == 5 and args.policies:
+        run_policy_comparison(args)
         return
 
     if args.config == 5:

@@ -43,7 +43,7 @@ class TraceRun:
     """Pool, allocator and device buffers for one replay of the trace."""
 
     def __init__(self, iterations: int = 200, seed: int = W.SEED_BASE + 5, shape=W.SHAPE_8B, device: int = 0,
-                 pool_factor: float = 1.25):
+                 pool_factor: float = 1.25, token_budget: int = 8192, chunk: int = 512):
         import torch
         self.torch = torch
         self.iterations = iterations
@@ -51,7 +51,8 @@ class TraceRun:
         self.shape = shape
         self.device = device
         self.requests = W.trace_arrivals(seed, iterations)
-        self.peak_pages = W.trace_peak_pages(self.requests, iterations=iterations)
+        self.policy = {"token_budget": int(token_budget), "chunk": int(chunk)}     # the fixed scheduler's two knobs
+        self.peak_pages = W.trace_peak_pages(self.requests, iterations=iterations, **self.policy)
         self.num_pages = max(16, int(math.ceil(pool_factor * self.peak_pages)))
         hq, hkv, d = shape
         dev = f"cuda:{device}"
@@ -80,7 +81,7 @@ class TraceRun:
         hq, hkv, d = self.shape
         rng = W.make_rng(self.seed + 1)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for it in W.fcfs_trace(self.requests, self._alloc, self._free, iterations=self.iterations):
+        for it in W.fcfs_trace(self.requests, self._alloc, self._free, iterations=self.iterations, **self.policy):
             n = int(it.q_lens.sum())
             if n == 0:
                 yield TraceStep(it.index, it.q_lens, it.ctx_lens, it.block_tables, None, None, None, None, None,

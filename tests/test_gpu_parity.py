@@ -308,14 +308,16 @@ def test_host_buffer_iteration_matches_device_path():
     run.close()
 
 
-def test_config5_trace_parity():
-    """Workload-shift trace (shortened to 80 iterations, across the rate switch at 50): pages come
-    from the library's allocator and are freed per request; the pool must match the oracle's bit
-    for bit at the end, and sampled attention outputs every iteration must be in tolerance."""
+@pytest.mark.parametrize("budget,chunk", [(8192, 512), (2048, 256)], ids=["budget8192_chunk512", "budget2048_chunk256"])
+def test_config5_trace_parity(budget, chunk):
+    """Workload-shift trace (shortened to 80 iterations, across the rate switch at 50), under the
+    configuration's scheduler and under a second fixed policy: pages come from the library's
+    allocator and are freed per request; the pool must match the oracle's bit for bit at the end,
+    and sampled attention outputs every iteration must be in tolerance."""
     import oracle
     from harness import compare_outputs
     from paper_2604_07144_b200.trace_runner import TraceRun
-    run = TraceRun(iterations=80)
+    run = TraceRun(iterations=80, token_budget=budget, chunk=chunk)
     hq, hkv, d = run.shape
     k_ref = np.full((run.num_pages, hkv, 16, d), W.CANARY, np.uint16)
     v_ref = k_ref.copy()

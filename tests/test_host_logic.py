@@ -275,6 +275,39 @@ def test_plan_predict_matches_the_cost_model_oracle():
     assert steps[1] < 0.95 * steps[0]
 
 
+def test_execution_model_matches_its_oracle_and_the_papers_table():
+    """paper_2604_07144_b200.execution_model against the oracle's term-by-term sum on random interval
+    lists, and against the paper's printed artifact-feedback rows."""
+    from oracle import execution_model as E
+    from paper_2604_07144_b200 import execution_model as M
+    from test_oracle_pins import _artifact_rows, _split
+    rng = np.random.default_rng(2)
+    for _ in range(50):
+        n = int(rng.integers(1, 8))
+        ivs = [M.Interval(*rng.random(4).tolist()) for _ in range(n)]
+        ref = E.t_total([i.t_sched for i in ivs], [i.t_stale for i in ivs], [i.t_reconfig for i in ivs],
+                        [i.t_serve for i in ivs])
+        assert np.isclose(M.total_time(ivs), ref, rtol=1e-12)
+    for name, n, stale, reconf, serve, total in _artifact_rows():
+        serve_parts = _split(rng, serve, n + 1)
+        ivs = [M.Interval(t_serve=serve_parts[0])] + [
+            M.Interval(t_sched=5.0, t_stale=a, t_reconfig=b, t_serve=c)
+            for a, b, c in zip(_split(rng, stale, n), _split(rng, reconf, n), serve_parts[1:])]
+        fb = M.artifact_feedback(ivs)
+        assert fb["N"] == n and abs(fb["T_total"] - total) < 0.05
+        assert abs(fb["sum_t_stale"] - stale) < 1e-9 and abs(fb["sum_t_reconfig"] - reconf) < 1e-9
+        assert abs(fb["sum_t_serve"] - serve) < 1e-9
+    # measured iterations grouped into intervals
+    times = [0.1] * 10
+    ivs = M.intervals_from_iterations(times, reschedule_at=[4, 7], t_sched_first=0.5, t_stale=[1.0, 2.0],
+                                      t_reconfig=[3.0])
+    assert [round(i.t_serve, 6) for i in ivs] == [0.4, 0.3, 0.3]
+    assert np.isclose(M.total_time(ivs), 0.5 + 1.0 + 1.0 + 2.0 + 3.0)
+    assert M.artifact_feedback(M.intervals_from_iterations(times))["N"] == 0
+    with pytest.raises(ValueError):
+        M.intervals_from_iterations(times, reschedule_at=[5, 3])
+
+
 def test_empty_batch_plans_to_nothing():
     pool = host_pool()
     p = ap.plan_create(pool, [], [], np.zeros((0, 1), np.int32), 8)

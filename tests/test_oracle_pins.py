@@ -263,6 +263,40 @@ def pin_page_copy_migration():
     assert oracle.copy_pages(k2, v2, k, v, [], []) == 0
 
 
+def _artifact_rows():
+    path = os.path.join(os.path.dirname(__file__), "golden", "table_artifact_feedback.txt")
+    rows = []
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            name, n, stale, reconf, serve, total = line.split()
+            rows.append((name, int(n), float(stale), float(reconf), float(serve), float(total)))
+    assert len(rows) == 3
+    return rows
+
+
+def _split(rng, total, parts):
+    """`parts` non-negative numbers adding up to `total`."""
+    w = rng.random(parts) + 0.1
+    return (w / w.sum() * total).tolist()
+
+
+def test_execution_model_oracle_reproduces_the_papers_table():
+    """Eq. "ttotal" against the printed rows: however the accumulated costs are spread over the
+    N reschedulings, the total is the printed T_total; dropping a term is noticed."""
+    from oracle import execution_model as E
+    rng = np.random.default_rng(1)
+    for name, n, stale, reconf, serve, total in _artifact_rows():
+        for _ in range(5):
+            t_serve = _split(rng, serve, n + 1)
+            t_stale = [123.0] + _split(rng, stale, n)            # entry 0 does not exist in the model
+            t_reconf = [456.0] + _split(rng, reconf, n)
+            t_sched = [0.0] + [9.9] * n                          # later scheduling time is t_stale, not added again
+            assert abs(E.t_total(t_sched, t_stale, t_reconf, t_serve) - total) < 0.05, name
+            assert abs(E.t_total(t_sched, t_stale, [0.0] * (n + 1), t_serve) - total) > 1.0, name
+    assert E.t_total([], [], [], []) == 0.0
+    assert E.t_total([2.0], [7.0], [7.0], [3.0]) == 5.0          # cold start only: scheduling + serving
+
+
 def test_roofline_model_pins():
     """The cost-model oracle (App. B Eq. "roofline") against what the mathematics fixes."""
     from oracle import roofline_model as R
