@@ -156,6 +156,44 @@ struct TimedScope {
 
 }  // namespace
 
+namespace ap {
+
+// The attention kernels of a plan, in the plan's dispatch mode.  Shared by every entry point that
+// runs attention; allocates nothing (the second stream and the events belong to the pool).
+cudaError_t launch_attention_kernels(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
+                                     float *o_part, float *lse_part, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+    if (plan->side_by_side) {
+        // Decode goes first, on the caller's stream, so that its few CTAs are resident when the
+        // prefill kernel's units (second stream, lower priority) fill the remaining SMs; as decode
+        // CTAs retire, prefill units take their SMs too.  The caller's stream continues after both.
+        e = cudaEventRecord(pool->fork_event, st);
+        if (e == cudaSuccess) {
+            TimedScope timed(pool, AP_KERNEL_DECODE, st);
+            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+        }
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pool->side_stream, pool->fork_event, 0);
+        if (e == cudaSuccess) {
+            TimedScope timed(pool, AP_KERNEL_PREFILL, pool->side_stream);
+            e = launch_prefill(pool, plan, q, out, lse, pool->side_stream);
+        }
+        if (e == cudaSuccess) e = cudaEventRecord(pool->join_event, pool->side_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, pool->join_event, 0);
+    } else {
+        if (plan->info.decode_items > 0) {
+            TimedScope timed(pool, AP_KERNEL_DECODE, st);
+            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
+        }
+        if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
+            TimedScope timed(pool, AP_KERNEL_PREFILL, st);
+            e = launch_prefill(pool, plan, q, out, lse, st);
+        }
+    }
+    return e;
+}
+
+}  // namespace ap
+
 extern "C" {
 
 const char *ap_status_string(int status) {
@@ -768,33 +806,7 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
     cudaStream_t st = (cudaStream_t)stream;
     float *o_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.o_part_off) : nullptr;
     float *lse_part = plan->ws.bytes ? (float *)((char *)workspace + plan->ws.lse_part_off) : nullptr;
-    cudaError_t e = cudaSuccess;
-    if (plan->side_by_side) {
-        // Decode goes first, on the caller's stream, so that its few CTAs are resident when the
-        // prefill kernel's units (second stream, lower priority) fill the remaining SMs; as decode
-        // CTAs retire, prefill units take their SMs too.  The caller's stream continues after both.
-        e = cudaEventRecord(pool->fork_event, st);
-        if (e == cudaSuccess) {
-            TimedScope timed(pool, AP_KERNEL_DECODE, st);
-            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-        }
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(pool->side_stream, pool->fork_event, 0);
-        if (e == cudaSuccess) {
-            TimedScope timed(pool, AP_KERNEL_PREFILL, pool->side_stream);
-            e = launch_prefill(pool, plan, q, out, lse, pool->side_stream);
-        }
-        if (e == cudaSuccess) e = cudaEventRecord(pool->join_event, pool->side_stream);
-        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, pool->join_event, 0);
-    } else {
-        if (plan->info.decode_items > 0) {
-            TimedScope timed(pool, AP_KERNEL_DECODE, st);
-            e = launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-        }
-        if (e == cudaSuccess && plan->info.prefill_tiles > 0) {
-            TimedScope timed(pool, AP_KERNEL_PREFILL, st);
-            e = launch_prefill(pool, plan, q, out, lse, st);
-        }
-    }
+    const cudaError_t e = ap::launch_attention_kernels(pool, plan, q, out, lse, o_part, lse_part, st);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return e == cudaErrorNotSupported ? AP_ERR_UNSUPPORTED : AP_ERR_CUDA;

@@ -139,6 +139,10 @@ cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, co
                                  float *lse, float *o_part, float *lse_part, cudaStream_t stream);
 cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                            float *lse, cudaStream_t stream);
+// Decode and prefill kernels of a plan: one after the other on `stream`, or, for a side-by-side plan,
+// decode on `stream` and prefill on the pool's second stream, joined back into `stream`.
+cudaError_t launch_attention_kernels(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
+                                     float *o_part, float *lse_part, cudaStream_t stream);
 // d_pairs: device [n_pairs][2] = (destination page, source page)
 cudaError_t launch_kv_copy_pages(const ap_kv_pool *dst_pool, const ap_kv_pool *src_pool, const int32_t *d_pairs,
                                  int n_pairs, cudaStream_t stream);

@@ -59,9 +59,7 @@ int ap_attention_iteration_static(ap_kv_pool *pool, const ap_plan *plan, const v
         // from an earlier call is ever read and nothing needs clearing.
         float *o_part = plan->ws.bytes ? (float *)((char *)ws + plan->ws.o_part_off) : nullptr;
         float *lse_part = plan->ws.bytes ? (float *)((char *)ws + plan->ws.lse_part_off) : nullptr;
-        cudaError_t e = cudaSuccess;
-        if (plan->info.decode_items > 0) e = ap::launch_decode_splitk(pool, plan, q, out, lse, o_part, lse_part, st);
-        if (e == cudaSuccess && plan->info.prefill_tiles > 0) e = ap::launch_prefill(pool, plan, q, out, lse, st);
+        const cudaError_t e = ap::launch_attention_kernels(pool, plan, q, out, lse, o_part, lse_part, st);
         if (e != cudaSuccess) {
             (void)cudaGetLastError();
             rc = e == cudaErrorNotSupported ? AP_ERR_UNSUPPORTED : AP_ERR_CUDA;

@@ -75,6 +75,22 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
         b.close()
 
 
+def test_static_workspace_with_a_mixed_plan_run_side_by_side():
+    # A plan whose decode part runs beside its prefill part (forced here) takes the same route
+    # through the library's own scratch: the pool's second stream and events already exist, so
+    # this entry point still allocates nothing.
+    batch = W._assemble("static_ws_mixed", W.SHAPE_8B, W.make_rng(904), np.array([140, 1, 1, 1], np.int32),
+                        np.array([500, 9000, 4000, 33], np.int32), 1.3)
+    run = GpuRun(batch, side_by_side=3)
+    try:
+        assert run.info["side_by_side"] == 1 and run.info["merge_entries"] > 0
+        ref = _reference(run)
+        _same(_static(run), ref)
+        _same(_static(run), ref)
+    finally:
+        run.close()
+
+
 def test_static_workspace_small_plan_and_argument_checks():
     # A plan with no cut stream needs no scratch at all and must work too; bad
     # arguments are refused before anything is launched.  (A plan larger than
