@@ -125,6 +125,22 @@ __host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool b_mn_major)
            ((uint32_t)(m >> 4) << 24);
 }
 
+// O (this thread's row, D fp32 columns in tensor memory) *= alpha.  Rare (the reference maximum moves
+// by more than the threshold only in a row's first steps), so it is kept out of line: the softmax loop
+// stays short and its registers are not shared with this path.
+template <int D>
+__device__ __noinline__ void rescale_o(uint32_t taddr, float alpha) {
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+        uint32_t oreg[32];
+        tmem_ld_32x32b_x32(taddr + c * 32, oreg);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
+        tmem_st_32x32b_x32(taddr + c * 32, oreg);
+    }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
@@ -347,17 +363,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 if (rescale) {
                     alpha = exp2_approx((m_used - m_new) * scale_log2);   // 0 on the first step
                     m_used = m_new;
-                    if (j > 0) {
-#pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t oreg[32];
-                            tmem_ld_32x32b_x32(lane_addr + col_o + c * 32, oreg);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) oreg[i] = __float_as_uint(__uint_as_float(oreg[i]) * alpha);
-                            tmem_st_32x32b_x32(lane_addr + col_o + c * 32, oreg);
-                        }
-                    }
+                    if (j > 0) rescale_o<D>(lane_addr + col_o, alpha);
                 }
                 const float ms = m_used * scale_log2;
                 const float2 sc2 = make_float2(scale_log2, scale_log2), nms2 = make_float2(-ms, -ms);
