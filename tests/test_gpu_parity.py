@@ -245,6 +245,35 @@ def test_plan_predict_tracks_the_measured_step(config):
         run.close()
 
 
+def test_page_copy_more_pairs_than_one_grid_dimension():
+    """70,000 pairs in one call (the launch is sliced at 65,535 pairs per grid): every destination page
+    must hold its source page, checked with torch on the device and on a sample against the oracle."""
+    import torch
+    import oracle
+    n, hkv, d = 70000, 2, 64
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    k1 = torch.randint(-32768, 32767, (n, hkv, 16, d), dtype=torch.int16, device="cuda", generator=gen).view(torch.bfloat16)
+    v1 = torch.randint(-32768, 32767, (n, hkv, 16, d), dtype=torch.int16, device="cuda", generator=gen).view(torch.bfloat16)
+    k2, v2 = torch.zeros_like(k1), torch.zeros_like(v1)
+    src_pool = ap.kv_pool_create(n, hkv, d, k1, v1)
+    dst_pool = ap.kv_pool_create(n, hkv, d, k2, v2)
+    rng = np.random.default_rng(9)
+    dst, src = rng.permutation(n).astype(np.int32), rng.integers(0, n, size=n).astype(np.int32)
+    ap.kv_copy_pages(dst_pool, src_pool, dst, src)
+    assert ap.last_device_status(dst_pool) == 0
+    di, si = torch.from_numpy(dst.astype(np.int64)).cuda(), torch.from_numpy(src.astype(np.int64)).cuda()
+    assert torch.equal(k2.view(torch.int16)[di], k1.view(torch.int16)[si])
+    assert torch.equal(v2.view(torch.int16)[di], v1.view(torch.int16)[si])
+    # the last pairs (second slice) once more against the oracle's copy
+    tail = slice(n - 300, n)
+    k_ref = np.zeros((n, hkv, 16, d), np.uint16)
+    v_ref = np.zeros_like(k_ref)
+    assert oracle.copy_pages(k_ref, v_ref, to_bits(k1), to_bits(v1), dst[tail], src[tail]) == 0
+    assert np.array_equal(to_bits(k2)[dst[tail]], k_ref[dst[tail]]) and np.array_equal(to_bits(v2)[dst[tail]], v_ref[dst[tail]])
+    ap.kv_pool_destroy(src_pool)
+    ap.kv_pool_destroy(dst_pool)
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]
