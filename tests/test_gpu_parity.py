@@ -282,6 +282,18 @@ def test_prefill_chunk_shapes():
         check_batch_full(b)
 
 
+def test_prefill_long_prefix_and_maximum_chunk():
+    """The largest prefill work the configurations allow: a chunk deep inside a long context (485 key
+    steps per unit, the K/V ring wraps ~190 times) and a whole 8192-token prompt in one iteration (the
+    token budget), at the 70B and 8B shapes; sampled outputs against the oracle."""
+    b = W._assemble("prefill_long_prefix", W.SHAPE_70B, W.make_rng(310), np.array([2048, 1], np.int32),
+                    np.array([60000 + 2048, 70001], np.int32), 1.05)
+    check_batch_sampled(b, 96, seed=1)
+    b = W._assemble("prefill_whole_budget", W.SHAPE_8B, W.make_rng(311), np.array([8192], np.int32),
+                    np.array([8192], np.int32), 1.05)
+    check_batch_sampled(b, 96, seed=2)
+
+
 def test_empty_and_skipped_sequences():
     b = W._assemble("skipped", W.SHAPE_S1, W.make_rng(400), np.array([0, 1, 0], np.int32), np.array([33, 70, 5], np.int32), 1.3)
     check_batch_full(b)
