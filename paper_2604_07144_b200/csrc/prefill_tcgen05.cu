@@ -259,11 +259,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     const uint32_t a0 = q_lo + (uint32_t)((x * Cfg::kQBytes) >> 4);
                     const uint32_t b0 = k_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColS + x * 128;
+                    // 16 elements of d per MMA: 32 bytes further inside the 64-element half, next half every four
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        umma_ss(leader, d, a0 + (uint32_t)(((ks >> 2) * (kTileM * 128) + (ks & 3) * 32) >> 4), q_hi,
-                                  b0 + (uint32_t)(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4), k_hi, kIdescQK,
-                                  ks > 0 ? 1u : 0u);
+                    for (int kh = 0; kh < D / 64; ++kh)
+                        umma_ss_x4(leader, d, a0 + (uint32_t)((kh * (kTileM * 128)) >> 4), q_hi,
+                                   b0 + (uint32_t)((kh * 1024) >> 4), k_hi, kIdescQK, kh > 0 ? 1u : 0u, 32u >> 4, 32u >> 4);
                     umma_commit(leader, &s_full[x]);
                 };
                 // O_x += P_x V with V in ring slot `slot`.  P: bf16 pairs in the first 64 columns of S_x
@@ -271,16 +271,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 auto issue_pv = [&](int x, int slot, bool first_step) {
                     const uint32_t b0 = v_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
                     const uint32_t d = tmem + Cfg::kColO + x * 128, a = tmem + Cfg::kColS + x * 128;
-                    if (!first_step) {
+                    constexpr uint32_t kVStep = (uint32_t)((2 * 1024 * Cfg::kHalves) >> 4);   // 16 keys of V
 #pragma unroll
-                        for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts(leader, d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV, 1u);
-                    } else {
-#pragma unroll
-                        for (int ks = 0; ks < kTileN / 16; ++ks)
-                            umma_ts(leader, d, a + ks * 8, b0 + (uint32_t)((ks * 2 * 1024 * Cfg::kHalves) >> 4), v_hi, kIdescPV,
-                                      ks > 0 ? 1u : 0u);
-                    }
+                    for (int kq = 0; kq < kTileN / 64; ++kq)
+                        umma_ts_x4(leader, d, a + kq * 32, b0 + kq * 4 * kVStep, v_hi, kIdescPV,
+                                   (first_step && kq == 0) ? 0u : 1u, 8u, kVStep);
                 };
                 if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag);
                 if (ok) {

@@ -211,6 +211,67 @@ __device__ __forceinline__ void umma_ts(uint32_t leader, uint32_t d_tmem, uint32
         : "memory");
 }
 
+// Four MMAs in one block: operand k is (a_lo + k * a_step, b_lo + k * b_step); the first one
+// accumulates only if `accumulate_first`, the others always.  One leader / accumulate predicate set-up
+// serves all four.
+__device__ __forceinline__ void umma_ss_x4(uint32_t leader, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                           uint32_t b_hi, uint32_t idesc, uint32_t accumulate_first, uint32_t a_step,
+                                           uint32_t b_step) {
+    asm volatile(
+        "{\n\t.reg .pred p, q, t;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 q, %7, 0;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "setp.eq.u32 t, 0, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t"
+        "add.u32 al, %1, %8;\n\t"
+        "add.u32 bl, %3, %9;\n\t"
+        "mov.b64 da, {al, %2};\n\t"
+        "mov.b64 db, {bl, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, t;\n\t"
+        "add.u32 al, al, %8;\n\t"
+        "add.u32 bl, bl, %9;\n\t"
+        "mov.b64 da, {al, %2};\n\t"
+        "mov.b64 db, {bl, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, t;\n\t"
+        "add.u32 al, al, %8;\n\t"
+        "add.u32 bl, bl, %9;\n\t"
+        "mov.b64 da, {al, %2};\n\t"
+        "mov.b64 db, {bl, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, t;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "r"(leader),
+          "r"(a_step), "r"(b_step)
+        : "memory");
+}
+
+// The same with A in tensor memory: operand k is (a_tmem + k * a_step, b_lo + k * b_step).
+__device__ __forceinline__ void umma_ts_x4(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate_first, uint32_t a_step, uint32_t b_step) {
+    asm volatile(
+        "{\n\t.reg .pred p, q, t;\n\t.reg .b64 db;\n\t.reg .b32 al, bl;\n\t"
+        "setp.ne.b32 q, %6, 0;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.eq.u32 t, 0, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t"
+        "add.u32 al, %1, %7;\n\t"
+        "add.u32 bl, %2, %8;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [al], db, %4, t;\n\t"
+        "add.u32 al, al, %7;\n\t"
+        "add.u32 bl, bl, %8;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [al], db, %4, t;\n\t"
+        "add.u32 al, al, %7;\n\t"
+        "add.u32 bl, bl, %8;\n\t"
+        "mov.b64 db, {bl, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [al], db, %4, t;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "r"(leader), "r"(a_step),
+          "r"(b_step)
+        : "memory");
+}
+
 // mbarrier arrives once all tcgen05.mma issued so far by the elected lane have completed
 __device__ __forceinline__ void umma_commit(uint32_t leader, uint64_t *bar) {
     asm volatile(
