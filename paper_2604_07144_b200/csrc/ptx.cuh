@@ -181,36 +181,11 @@ __device__ __forceinline__ uint32_t elect_one() {
     return pred;
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate.  The 64-bit shared-memory
-// descriptors are given as (low, high) words: the high word (stride offset, version, layout) is
-// constant per operand and only the low word (address, leading offset) moves, so one 32-bit add per
-// operand and MMA is enough.  Executed by the whole warp; the lane with `leader` != 0 issues.
-__device__ __forceinline__ void umma_ss(uint32_t leader, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
-                                        uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %2};\n\t"
-        "mov.b64 db, {%3, %4};\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "setp.ne.b32 q, %7, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
-        : "memory");
-}
-
-// D[tmem] (+)= A[tmem] * B[smem desc]
-__device__ __forceinline__ void umma_ts(uint32_t leader, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
-                                        uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "setp.ne.b32 q, %6, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(leader)
-        : "memory");
-}
-
+// tcgen05.mma, kind::f16 (bf16 inputs, fp32 accumulate): D[tmem] (+)= A * B with A from shared memory
+// (`ss`) or tensor memory (`ts`) and B from shared memory.  The 64-bit shared-memory descriptors are
+// given as (low, high) words: the high word (stride offset, version, layout) is constant per operand
+// and only the low word (address, leading offset) moves.  Executed by the whole warp; the lane with
+// `leader` != 0 issues.
 // Four MMAs in one block: operand k is (a_lo + k * a_step, b_lo + k * b_step); the first one
 // accumulates only if `accumulate_first`, the others always.  One leader / accumulate predicate set-up
 // serves all four.
