@@ -38,6 +38,11 @@
  *     followed by ap_attention_iteration on the same stream needs no sync.
  *   - A plan must outlive the launches that use it (destroy it after the stream
  *     has passed them, or after ap_last_device_status).
+ *   - A pool and its plans are not thread-safe: calls that name the same pool must
+ *     come from one host thread at a time (the pool owns staging buffers, a second
+ *     stream with its fork / join events, and the allocator state).  Different pools
+ *     are independent.  Launches of one pool on different streams that may overlap
+ *     on the GPU are not supported either: they share the split-K arrival counters.
  */
 #ifndef AP_SERVING_H
 #define AP_SERVING_H
