@@ -274,6 +274,52 @@ def test_page_copy_more_pairs_than_one_grid_dimension():
     ap.kv_pool_destroy(dst_pool)
 
 
+def _shared_prefix_batch():
+    """Three sequences reading the same six prefix pages (96 tokens) through their block tables: two
+    decode rows and a prefill chunk; every sequence appends into pages of its own."""
+    b = W._assemble("shared_prefix", W.SHAPE_8B, W.make_rng(61), np.array([1, 1, 40], np.int32),
+                    np.array([300, 180, 96 + 40], np.int32), 1.3)
+    b.block_tables[1, :6] = b.block_tables[0, :6]
+    b.block_tables[2, :6] = b.block_tables[0, :6]
+    return b
+
+
+def test_shared_prefix_pages_are_read_by_several_sequences():
+    check_batch_full(_shared_prefix_batch())
+
+
+def test_fork_a_sequence_with_copy_on_write_of_its_last_page():
+    """A sequence is forked: the fork's block table names the parent's full pages and a fresh page that
+    ap_kv_copy_pages fills from the parent's partly filled last page; then parent and fork each append a
+    different token and attend.  Against the oracle doing the same copy, append and attention."""
+    import oracle
+    from harness import compare_outputs
+    base = W._assemble("fork_parent", W.SHAPE_8B, W.make_rng(62), np.array([1, 1], np.int32),
+                       np.array([301, 301], np.int32), 1.5)          # row 1 is only a donor of pages and tokens
+    n_pages = (301 + 15) // 16
+    parent = base.block_tables[0, :n_pages].copy()
+    fresh = int(base.block_tables[1, 0])                           # a page the parent does not use
+    fork = parent.copy()
+    fork[-1] = fresh
+    base.block_tables[1, :n_pages] = fork
+    run = GpuRun(base)
+    try:
+        k_ref, v_ref = base.k_pool.copy(), base.v_pool.copy()
+        ap.kv_copy_pages(run.pool, run.pool, [fresh], [int(parent[-1])])
+        assert oracle.copy_pages(k_ref, v_ref, k_ref, v_ref, [fresh], [int(parent[-1])]) == 0
+        run.append()
+        run.attend()
+        assert run.status() == 0
+        assert oracle.kv_append(k_ref, v_ref, base.q_lens, base.ctx_lens, base.block_tables, base.k_new, base.v_new) == 0
+        assert np.array_equal(to_bits(run.k_pool), k_ref) and np.array_equal(to_bits(run.v_pool), v_ref)
+        ref_out, ref_lse = oracle.attention(k_ref, v_ref, base.q_lens, base.ctx_lens, base.block_tables, base.q)
+        compare_outputs(to_bits(run.out)[:2], run.lse.cpu().numpy()[:2], ref_out, ref_lse, "fork")
+        # same history, different new token and query: the two rows must differ
+        assert not np.array_equal(to_bits(run.out)[0], to_bits(run.out)[1])
+    finally:
+        run.close()
+
+
 def test_prefill_chunk_shapes():
     # whole prompt, chunk on a prefix, ragged last tile, several tiles, page-misaligned prefix
     cases = [([128], [128]), ([1 + 128], [129]), ([200], [777]), ([300], [300]), ([37], [1000]), ([512], [4096 + 512])]

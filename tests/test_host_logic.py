@@ -308,6 +308,22 @@ def test_execution_model_matches_its_oracle_and_the_papers_table():
         M.intervals_from_iterations(times, reschedule_at=[5, 3])
 
 
+def test_shared_pages_may_be_read_but_not_appended_to_twice():
+    """Block tables may name the same page in several sequences as long as no slot is written by two of
+    them: a shared read-only prefix plans fine, two sequences appending into the same slot are refused."""
+    b = W._assemble("shared", W.SHAPE_S1, W.make_rng(71), np.array([1, 1], np.int32), np.array([100, 100], np.int32), 1.3,
+                    with_pool=False)
+    pool = ap.kv_pool_create(b.num_pages, b.num_kv_heads, b.head_dim, device=-1)
+    bt = b.block_tables.copy()
+    bt[1, :6] = bt[0, :6]                                   # positions 0..95 shared, position 99 in own pages
+    ap.plan_destroy(ap.plan_create(pool, b.q_lens, b.ctx_lens, bt, b.num_q_heads))
+    bt[1, 6] = bt[0, 6]                                     # now both append position 99 into the same slot
+    with pytest.raises(ap.ApError) as e:
+        ap.plan_create(pool, b.q_lens, b.ctx_lens, bt, b.num_q_heads)
+    assert e.value.status == B.AP_ERR_BAD_BLOCK_TABLE
+    ap.kv_pool_destroy(pool)
+
+
 def test_empty_batch_plans_to_nothing():
     pool = host_pool()
     p = ap.plan_create(pool, [], [], np.zeros((0, 1), np.int32), 8)
