@@ -1,16 +1,21 @@
 #!/usr/bin/env python
 """Benchmark of the paged-KV serving iteration (KV append + GQA attention).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2|3|4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2|3|4|5]
 
 A step is one pass of the whole hot path over one synthetic batch: KV append,
 split-K decode attention, LSE merge and (for batches with prefill chunks)
-prefill attention.  The default workload is the decode-heavy ragged batch on
-the Llama-3-8B attention shape (64 sequences, contexts log-uniform in
-128..8192).  Prints ONE JSON line (rank 0).
+prefill attention.  The headline workload (`value`) is the decode-heavy ragged
+batch on the Llama-3-8B attention shape (64 sequences, contexts log-uniform in
+128..8192).  Without --config the same run also times the mixed iteration
+(both dispatch modes), the long-context decode and the workload-shift trace and
+reports them under `configs`, so that the HBM-bound and the tensor-bound kernel
+each have a measured roofline fraction in the one line.  Prints ONE JSON line
+(rank 0).
 
-Timing: CUDA events on the launching stream around exactly K steps after W
-warm-up steps, barrier + synchronize on both sides, max over ranks.  Every
+Timing: CUDA events on the launching stream around K steps (repeated back to
+back until the region lasts about a second, so that clock samples fall inside it)
+after W warm-up steps, barrier + synchronize on both sides, max over ranks.  Every
 step reads a different copy of the KV pool (rotation among copies whose
 combined size is many times the L2), so KV reads are cold.  The plan (host
 work list + one H2D copy) is built once per batch outside `value`'s timed
@@ -38,20 +43,17 @@ sys.path.insert(0, ROOT)
 METRIC = "serving_iteration_attention_kv_tokens_per_s"
 UNIT = "KV-tokens/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitk launch on the
-# bench workload (ncu capture summarised under profiles/), keyed by the hash of
-# the kernel's source file (decode_splitk.cu) the counters were taken from; a changed kernel reports null.
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of a kernel on a bench
+# workload (ncu captures summarised under profiles/), keyed by (kernel, config, hash of
+# the kernel's source file the counters were taken from); a changed kernel reports null.
 NCU_TRAFFIC = {
-    # profiles/decode_splitk_config2.md: 536.9 MB read + 5.3 MB written per launch (algorithmic 535.0 MB)
-    (2, "04f79039326158ed"): 542.2e6,
 }
 
 
-def kernel_source_hash() -> str:
+def kernel_source_hash(source_file: str) -> str:
     h = hashlib.sha256()
-    for f in ("decode_splitk.cu",):
-        with open(os.path.join(ROOT, "paper_2604_07144_b200", "csrc", f), "rb") as fh:
-            h.update(fh.read())
+    with open(os.path.join(ROOT, "paper_2604_07144_b200", "csrc", source_file), "rb") as fh:
+        h.update(fh.read())
     return h.hexdigest()[:16]
 
 
@@ -297,7 +299,7 @@ def run_trace_bench(args):
                        "kv_tokens": t, "device_ms": m, "kv_tokens_per_s": (t / (m * 1e-3) if m else None),
                        "new_tokens": sum(p[5] for p in sel)})
     rates = sorted(p[1] / (p[2] * 1e-3) for p in per_iter)
-    print(json.dumps({
+    return ({
         "metric": METRIC, "value": toks / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": len(per_iter),
         "warmup": iterations, "ms_per_step": ms / max(len(per_iter), 1), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -310,8 +312,8 @@ def run_trace_bench(args):
         "per_iteration_kv_tokens_per_s": {"min": rates[0], "median": rates[len(rates) // 2], "max": rates[-1]},
         "phases": phases,
         "kernels": {k: {"launches": n, "us_per_launch": (1e3 * m / n if n else None)} for k, (m, n) in kt.items()},
-        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
-    }))
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")} if clocks else None,
+    })
 
 
 def run_policy_comparison(args):
@@ -405,60 +407,21 @@ def run_page_copy_bench(args):
     ap.kv_pool_destroy(src)
 
 
-def main():
-    ap_ = argparse.ArgumentParser()
-    ap_.add_argument("--gpus", type=int, default=1)
-    ap_.add_argument("--steps", type=int, default=300)
-    ap_.add_argument("--warmup", type=int, default=10)
-    ap_.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap_.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5])
-    ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
-    ap_.add_argument("--no-cpu-baseline", action="store_true")
-    ap_.add_argument("--policies", action="store_true",
-                     help="with --config 5: replay the trace under several fixed scheduling policies (token budget, "
-                          "prefill chunk) and score each by the paper's trace completion time on measured iterations")
-    ap_.add_argument("--page-copy", action="store_true",
-                     help="time ap_kv_copy_pages on config 2's used pages instead of the serving iteration")
-    ap_.add_argument("--side-by-side", type=int, default=None,
-                     help="mixed iterations: 0 = decode then prefill, 1 = planner decides (library default), "
-                          "k >= 2 = decode on k CTAs next to prefill")
-    args = ap_.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+def measure_config(config: int, args, rank: int, world: int, local_rank: int, side_by_side=None, with_e2e=True,
+                   min_region_s: float = 1.0):
+    """Times one workload on this rank's GPU and returns every figure the JSON line carries for it.
 
-    if args.impl == "reference":
-        run_reference(args)
-        return
-
-    if args.page_copy:
-        run_page_copy_bench(args)
-        return
-
-    if args.config == 5 and args.policies:
-        run_policy_comparison(args)
-        return
-
-    if args.config == 5:
-        run_trace_bench(args)
-        return
-
+    Pass 1 (the timed region): `repeats` blocks of K steps, kernels back to back in the stream, no events
+    between them; `repeats` is chosen from the warm-up so that the region lasts at least min_region_s
+    (clock samples need a region much longer than the sampling period).  Pass 2: the same steps with a
+    CUDA-event pair around every kernel, for the per-kernel times.  Then the end-to-end loop through
+    ap_serving_iteration_host with pinned host buffers."""
     import torch
-    import torch.distributed as dist
     import paper_2604_07144_b200 as ap
     from paper_2604_07144_b200 import replicas
-    from paper_2604_07144_b200 import workloads as W
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    # replicas only: every rank serves its own independent batch, no data-path collective
-    batch = make_batch(args.config, seed_offset=rank)
+    batch = make_batch(config, seed_offset=rank)
     hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
 
     def dev_bf16(bits):
@@ -473,8 +436,8 @@ def main():
         kp, vp = (k0, v0) if c == 0 else (k0.clone(), v0.clone())
         k_planes.append(kp); v_planes.append(vp)
         pools.append(ap.kv_pool_create(batch.num_pages, hkv, d, kp, vp, device=local_rank))
-        if args.side_by_side is not None:
-            ap.kv_pool_set_side_by_side(pools[-1], args.side_by_side)
+        if side_by_side is not None:
+            ap.kv_pool_set_side_by_side(pools[-1], side_by_side)
         plans.append(ap.plan_create(pools[-1], batch.q_lens, batch.ctx_lens, batch.block_tables, hq))
     info = ap.plan_get_info(plans[0])
     q, k_new, v_new = dev_bf16(batch.q), dev_bf16(batch.k_new), dev_bf16(batch.v_new)
@@ -493,37 +456,41 @@ def main():
         replicas.barrier()
         torch.cuda.synchronize()
 
-    def reduce_max(x: float) -> float:
-        return replicas.reduce_max(x, dev)
+    reduce_max = lambda x: replicas.reduce_max(x, dev)
+    reduce_sum = lambda x: replicas.reduce_sum(x, dev)
 
-    def reduce_sum(x: float) -> float:
-        return replicas.reduce_sum(x, dev)
-
-    # ---- device-resident timing
-    for i in range(args.warmup):
+    # ---- warm-up, which also sizes the timed region
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(max(args.warmup - 3, 0)):
         step(i)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(3):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
     for p in pools:
         assert ap.last_device_status(p) == 0
+    est_ms = reduce_max(e0.elapsed_time(e1)) / 3
+    repeats = max(1, int(np.ceil(min_region_s * 1e3 / max(est_ms * args.steps, 1e-3))))
+    n_timed = args.steps * repeats
+
     sampler = ClockSampler(local_rank)
     barrier()
     if rank == 0:
         sampler.start()
-    # Pass 1, the timed region: K steps as a user runs them (kernels back to back in the stream).
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for i in range(args.steps):
+    for i in range(n_timed):
         step(i)
     e1.record()
     barrier()
     ms_total = reduce_max(e0.elapsed_time(e1))
-    # Pass 2: the same K steps with a CUDA-event pair around every kernel, for the per-kernel times
-    # (the events sit between the kernels, so this pass cannot overlap one kernel's launch with the
-    # tail of the one before; its step time is reported beside the first pass's).
     for p in pools:
         ap.profile_enable(p, True)
+    n_prof = args.steps * min(repeats, max(1, int(np.ceil(0.3e3 / max(est_ms * args.steps, 1e-3)))))
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record()
-    for i in range(args.steps):
+    for i in range(n_prof):
         step(i)
     e3.record()
     barrier()
@@ -537,7 +504,7 @@ def main():
         ap.profile_enable(p, False)
         assert ap.last_device_status(p) == 0
     total_tokens = reduce_sum(float(batch.kv_tokens))
-    ms_per_step = ms_total / args.steps
+    ms_per_step = ms_total / n_timed
     value = total_tokens / (ms_per_step * 1e-3)
 
     # ---- plan cost (host + upload), reported separately
@@ -548,47 +515,76 @@ def main():
     plan_ms = (time.perf_counter() - t0) / 20 * 1e3
 
     # ---- end to end through the host-buffer entry point
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
-    hq_, hk_, hv_ = pin(batch.q), pin(batch.k_new), pin(batch.v_new)
-    hout = torch.empty((batch.n_new, hq, d), dtype=torch.int16).pin_memory()
-    hlse = torch.empty((batch.n_new, hq), dtype=torch.float32).pin_memory()
+    e2e = None
+    if with_e2e:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        hq_, hk_, hv_ = pin(batch.q), pin(batch.k_new), pin(batch.v_new)
+        hout = torch.empty((batch.n_new, hq, d), dtype=torch.int16).pin_memory()
+        hlse = torch.empty((batch.n_new, hq), dtype=torch.float32).pin_memory()
 
-    def e2e_step(i):
-        ap.serving_iteration_host(pools[i % copies], batch.q_lens, batch.ctx_lens, batch.block_tables, hq,
-                                  hq_, hk_, hv_, hout, hlse)
+        def e2e_step(i):
+            ap.serving_iteration_host(pools[i % copies], batch.q_lens, batch.ctx_lens, batch.block_tables, hq,
+                                      hq_, hk_, hv_, hout, hlse)
 
-    e2e_steps = max(10, args.steps // 4)
-    for i in range(3):
-        e2e_step(i)
-    barrier()
-    e0.record()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    e1.record()
-    barrier()
-    e2e_ms = reduce_max(e0.elapsed_time(e1)) / e2e_steps
-    h2d = int(batch.q.nbytes + batch.k_new.nbytes + batch.v_new.nbytes)
-    d2h = int(hout.numel() * 2 + hlse.numel() * 4)
+        for i in range(3):
+            e2e_step(i)
+        barrier()
+        t0 = time.perf_counter()
+        e2e_step(0)
+        torch.cuda.synchronize()
+        est = (time.perf_counter() - t0) * 1e3
+        e2e_steps = max(10, min(n_timed, int(np.ceil(0.5e3 / max(est, 1e-3)))))
+        barrier()
+        e0.record()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        e1.record()
+        barrier()
+        e2e_ms = reduce_max(e0.elapsed_time(e1)) / e2e_steps
+        e2e = {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(batch.q.nbytes + batch.k_new.nbytes + batch.v_new.nbytes),
+               "d2h_bytes_per_step": int(hout.numel() * 2 + hlse.numel() * 4 + 4), "ms_per_step": e2e_ms,
+               "steps": e2e_steps,
+               "includes": "plan build + upload, H2D of q/k_new/v_new, append, attention, D2H of out/lse/status, sync"}
+        got = torch.from_numpy(hout.numpy().copy()).view(torch.bfloat16).float()
+        assert bool(torch.isfinite(got).all()) and bool(torch.isfinite(hlse).all())
 
     # sanity: the timed path produced finite numbers
     assert bool(torch.isfinite(out.float()).all()) and bool(torch.isfinite(lse).all())
 
+    res = None
     if rank == 0:
         peaks = measured_peaks()
         alg = algorithmic_bytes(batch, info)
-        dec_ms, dec_n = kt.get("decode_splitk", (0.0, 0))
+        kernels = {name: {"launches": n, "us_per_launch": (1e3 * ms / n if n else None)} for name, (ms, n) in kt.items()}
+        dec_us = kernels.get("decode_splitk", {}).get("us_per_launch")
+        pre_us = kernels.get("prefill", {}).get("us_per_launch")
+        fus_us = kernels.get("fused_mixed", {}).get("us_per_launch")
         # the profile sums cover this rank's launches only
-        achieved = alg["decode_kernel"] / (dec_ms / max(dec_n, 1) * 1e-3) / 1e9 if dec_n else 0.0
-        roofline = {
+        achieved = alg["decode_kernel"] / (dec_us * 1e-6) / 1e9 if dec_us else 0.0
+        decode_roofline = {
             "bound": "hbm", "kernel": "decode_splitk", "achieved": achieved, "peak": peaks["hbm_gbs"],
             "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-            "traffic": NCU_TRAFFIC.get((args.config, kernel_source_hash())),
-            "bytes_per_launch": alg["decode_kernel"], "us_per_launch": 1e3 * dec_ms / max(dec_n, 1),
+            "traffic": NCU_TRAFFIC.get(("decode_splitk", config, kernel_source_hash("decode_splitk.cu"))),
+            "bytes_per_launch": alg["decode_kernel"], "us_per_launch": dec_us,
             "frac_of_nominal_8TBs": achieved / 8000.0,
         }
-        if info["side_by_side"]:
-            roofline["note"] = (f"in this plan decode runs on {info['decode_ctas']} SMs next to the prefill kernel, so its own "
-                                "time is not a whole-GPU bandwidth figure; see step_roofline")
+        concurrent = bool(info["side_by_side"]) or bool(fus_us)
+        if concurrent:
+            decode_roofline["note"] = ("in this plan decode shares the GPU with prefill, so its own time is not a "
+                                       "whole-GPU bandwidth figure; see step_roofline")
+        prefill_roofline = None
+        if pre_us:
+            tf = alg["prefill_flops"] / (pre_us * 1e-6) / 1e12
+            prefill_roofline = {
+                "bound": "tensor", "kernel": "prefill_tcgen05", "achieved": tf, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": f"of {peaks['source']} (burst)",
+                "frac_of_sustained": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
+                "traffic": NCU_TRAFFIC.get(("prefill_tcgen05", config, kernel_source_hash("prefill_tcgen05.cu"))),
+                "flops_per_launch": alg["prefill_flops"], "us_per_launch": pre_us,
+            }
+            if concurrent:
+                prefill_roofline["note"] = "runs next to the decode kernel in this plan: not a whole-GPU figure"
         # whole step against the slower of its two bounds: all algorithmic bytes at the measured copy
         # bandwidth, all algorithmic flops at the measured bf16 peak
         t_bytes = alg["total"] / (peaks["hbm_gbs"] * 1e9)
@@ -598,29 +594,30 @@ def main():
                          "frac": max(t_bytes, t_flops) / (ms_per_step * 1e-3),
                          "note": "bound = max(bytes / copy bandwidth, flops / bf16 peak): reachable only if the "
                                  "HBM-bound and the tensor-bound parts overlap perfectly; sum = no overlap"}
-        kernels = {name: {"launches": n, "us_per_launch": (1e3 * ms / n if n else None)} for name, (ms, n) in kt.items()}
+        launches_per_step = info["launches_append"] + info["launches_attention"]
         res = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "value": value, "ms_per_step": ms_per_step, "steps": args.steps, "repeats": repeats, "timed_steps": n_timed,
+            "timed_ms": ms_total,
             "config": {"workload": batch.name, "num_q_heads": hq, "num_kv_heads": hkv, "head_dim": d,
                        "page_size": 16, "sequences": batch.batch, "new_tokens": batch.n_new,
                        "kv_tokens_per_step_per_gpu": batch.kv_tokens,
+                       "dispatch": ("fused" if fus_us else "side_by_side" if info["side_by_side"] else "sequential"),
                        "l2": f"rotation among {copies} pool copies ({copies * kv_bytes / 1e9:.2f} GB of KV, each step's "
                              f"{kv_bytes / 1e6:.0f} MB larger than the 126 MB L2)",
+                       "timed_region": f"{repeats} x {args.steps} steps back to back ({ms_total:.0f} ms), sized from the warm-up "
+                                       f"to last >= {min_region_s} s so the clock sampler sees it",
                        "parallelism": "replicas only (one independent batch per GPU, no collective)"},
-            "gpu_launches": int(sum(n for _, n in kt.values())),
-            "e2e": {"value": total_tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                    "includes": "plan build + upload, H2D of q/k_new/v_new, append, attention, D2H of out/lse, sync"},
+            "gpu_launches": int(n_timed * launches_per_step),
+            "e2e": e2e,
             "plan": {"host_ms": plan_ms, "in_value": False, "in_e2e": True, **{k: info[k] for k in (
                 "decode_items", "decode_ctas", "merge_entries", "prefill_tiles", "side_by_side")}},
-            "roofline": roofline,
+            "roofline": decode_roofline,
+            "prefill_roofline": prefill_roofline,
             "step_roofline": step_roofline,
             "kernels": kernels,
-            "kernel_timing": {"how": "second pass of the same K steps with a CUDA-event pair around every kernel, "
+            "kernel_timing": {"how": "second pass of the same steps with a CUDA-event pair around every kernel, "
                                      "right after the timed pass; the timed pass itself has no events between kernels",
-                              "ms_per_step_with_events": ms_total_profiled / args.steps},
+                              "steps": n_prof, "ms_per_step_with_events": ms_total_profiled / n_prof},
             "paper_model_us": {"decode_splitk": paper_model_us(alg["decode_flops"], alg["decode_kernel"], peaks),
                                "prefill": paper_model_us(alg["prefill_flops"], alg["prefill_kernel"], peaks),
                                "note": "T_op = F / min(F/A * B, F_peak) with this GPU's measured copy bandwidth and "
@@ -629,19 +626,120 @@ def main():
                               if k.endswith("_us")},
                            "note": "ap_plan_predict: roofline_* = the paper's operator model computed by the library, "
                                    "model_* = the planner's calibrated cost model; compare model_step_us with ms_per_step"},
-            "prefill_tflops": (alg["prefill_flops"] / (kernels["prefill"]["us_per_launch"] * 1e-6) / 1e12
-                               if kernels.get("prefill", {}).get("us_per_launch") else None),
+            "prefill_tflops": prefill_roofline["achieved"] if prefill_roofline else None,
             "step_gbs": alg["total"] / (ms_per_step * 1e-3) / 1e9,
-            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")} if clocks else None,
+            "clocks": ({**{k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+                        "ms_x_mhz": (ms_per_step * clocks["sm_mhz"] if clocks["sm_mhz"] else None)} if clocks else None),
         }
-        if world == 1 and not args.no_cpu_baseline:
-            res["cpu_baseline"] = cpu_oracle_baseline(batch)
-        print(json.dumps(res))
-
     for pl in plans:
         ap.plan_destroy(pl)
     for p in pools:
         ap.kv_pool_destroy(p)
+    del k_planes, v_planes, k0, v0, q, k_new, v_new, out, lse, ws
+    torch.cuda.empty_cache()
+    return res, batch
+
+
+def compact(res):
+    """The figures of one extra workload that go under `configs` in the JSON line."""
+    keep = ("value", "ms_per_step", "repeats", "timed_steps", "timed_ms", "gpu_launches", "kernels", "roofline",
+            "prefill_roofline", "prefill_tflops", "step_roofline", "step_gbs", "e2e", "clocks", "prediction")
+    out = {k: res[k] for k in keep if k in res}
+    out["workload"] = res["config"]["workload"]
+    out["dispatch"] = res["config"]["dispatch"]
+    out["plan"] = res["plan"]
+    for r in ("roofline", "prefill_roofline"):
+        if out.get(r):
+            out[r] = {k: v for k, v in out[r].items() if k not in ("note",)}
+    return out
+
+
+def main():
+    ap_ = argparse.ArgumentParser()
+    ap_.add_argument("--gpus", type=int, default=1)
+    ap_.add_argument("--steps", type=int, default=100)
+    ap_.add_argument("--warmup", type=int, default=10)
+    ap_.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap_.add_argument("--config", type=int, default=0, choices=[0, 2, 3, 4, 5],
+                     help="0 (default): config 2 is the headline value and configs 3 (both dispatch modes), 4 and the "
+                          "config-5 trace are timed in the same run and reported under `configs`; 2|3|4|5: that one only")
+    ap_.add_argument("--pool-copies", type=int, default=0, help="0 = enough copies for >= 2 GB of KV")
+    ap_.add_argument("--no-cpu-baseline", action="store_true")
+    ap_.add_argument("--min-region-s", type=float, default=1.0,
+                     help="the K steps are repeated until the timed region lasts at least this long")
+    ap_.add_argument("--policies", action="store_true",
+                     help="with --config 5: replay the trace under several fixed scheduling policies (token budget, "
+                          "prefill chunk) and score each by the paper's trace completion time on measured iterations")
+    ap_.add_argument("--page-copy", action="store_true",
+                     help="time ap_kv_copy_pages on config 2's used pages instead of the serving iteration")
+    ap_.add_argument("--side-by-side", type=int, default=None,
+                     help="mixed iterations: 0 = decode then prefill, 1 = planner decides (library default), "
+                          "k >= 2 = decode on k CTAs next to prefill")
+    args = ap_.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    all_configs = args.config == 0
+    if all_configs:
+        args.config = 2
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    if args.page_copy:
+        run_page_copy_bench(args)
+        return
+
+    if args.config == 5 and args.policies:
+        run_policy_comparison(args)
+        return
+
+    if args.config == 5:
+        print(json.dumps(run_trace_bench(args)))
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # replicas only: every rank serves its own independent batch, no data-path collective
+    res, batch = measure_config(args.config, args, rank, world, local_rank, side_by_side=args.side_by_side,
+                                min_region_s=args.min_region_s)
+    extras = {}
+    if all_configs and world == 1:
+        # the other roofline-bearing workloads, in the same process and on the same GPU
+        r3s, _ = measure_config(3, args, rank, world, local_rank, side_by_side=0, min_region_s=args.min_region_s)
+        extras["config3_sequential"] = compact(r3s)
+        r3, _ = measure_config(3, args, rank, world, local_rank, min_region_s=args.min_region_s)
+        extras["config3"] = compact(r3)
+        r4, _ = measure_config(4, args, rank, world, local_rank, min_region_s=args.min_region_s)
+        extras["config4"] = compact(r4)
+        t5 = run_trace_bench(args)
+        extras["config5"] = {k: t5[k] for k in ("value", "ms_per_step", "steps", "gpu_launches", "phases",
+                                                "per_iteration_kv_tokens_per_s", "kernels", "clocks")}
+        extras["config5"]["workload"] = t5["config"]["workload"]
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        }
+        line.update({k: v for k, v in res.items() if k not in ("value", "ms_per_step", "steps")})
+        if extras:
+            line["configs"] = extras
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_oracle_baseline(batch)
+        print(json.dumps(line))
+
     if world > 1:
         dist.destroy_process_group()
 

@@ -72,9 +72,9 @@ typedef struct ap_plan ap_plan;       /* opaque */
 
 /*
  * KV page pool (finite token capacity: App. B Eq. "oom", App. C.2).
- * k_base/v_base: device, each ap_kv_pool_bytes() long and 1024-byte aligned,
- * owned by the caller; or both NULL, then the library allocates (and zero
- * fills) and frees them.  head_dim is 64 or 128; page_size must be 16;
+ * k_base/v_base: device, each ap_kv_pool_bytes() long and 16-byte aligned
+ * (what a tensor map's base address needs), owned by the caller; or both NULL,
+ * then the library allocates (and zero fills) and frees them.  head_dim is 64 or 128; page_size must be 16;
  * num_q_heads / num_kv_heads may be 1..8 (given per batch).
  */
 typedef struct ap_pool_desc {
@@ -292,9 +292,10 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
  *    is rejected with AP_ERR_WORKSPACE_TOO_SMALL before anything is launched
  *    (4 MiB covers every plan the planner makes for 148 SMs at head_dim 128
  *    and 8 query heads per kv head, including 131072-token contexts).
- *  - The first call on each device looks up the array's device address (one
- *    runtime query, cached afterwards); make that first call outside any
- *    stream capture.
+ *  - The array's device address is looked up once per device when a pool is
+ *    created on it (ap_kv_pool_create, which allocates anyway and must not run
+ *    inside a stream capture); that is also when the runtime brings the array
+ *    into being on the device.  The call here only reads the cached address.
  *  - All calls on a device share the one array, and it keeps whatever the last
  *    call left in it.  Nothing has to start at zero: every partial is written
  *    in full before it is read within the same call.  Two calls that overlap
@@ -320,10 +321,35 @@ int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, cons
 
 /* Synchronises `stream` and returns (and clears) the device status word:
  * AP_OK, AP_ERR_BAD_BLOCK_TABLE (a kernel met an out-of-range page id) or
- * AP_ERR_TIMEOUT (a bounded wait inside a kernel ran out). */
+ * AP_ERR_TIMEOUT (a bounded wait inside a kernel ran out).  After an error it
+ * also clears the split-K arrival counters, which a kernel that gave up may
+ * have left raised, so the pool can be used again. */
 int ap_last_device_status(ap_kv_pool *pool, void *stream);
 
 const char *ap_status_string(int status);
+
+/*
+ * Bound of every wait inside the kernels (failure detection: Sec. 5.1 counts a
+ * stalled or failed serving plan as stale time, so a kernel must end and report
+ * rather than hang).  Every mbarrier wait in the attention kernels gives up
+ * after limit_ns nanoseconds on the GPU's global timer, records AP_ERR_TIMEOUT
+ * in the pool's status word and lets the kernel return; outputs of that launch
+ * are then undefined.  Default 2 s; limit_ns = 0 restores it.  Applies to
+ * launches made afterwards.
+ */
+int ap_kv_pool_set_wait_limit(ap_kv_pool *pool, uint64_t limit_ns);
+
+/*
+ * Self-test of that error path: queues a one-warp kernel on `stream` that
+ * waits, through the same bounded-wait routine the attention kernels use, on a
+ * barrier nothing ever arrives on.  It ends by itself after limit_ns
+ * (0 < limit_ns <= 2 s, else INVALID_ARG) and leaves AP_ERR_TIMEOUT in the
+ * pool's status word, which the next ap_last_device_status returns and clears.
+ * With leave_counter != 0 it also leaves one split-K arrival counter raised, as
+ * an attention kernel that gave up mid-stream would; ap_last_device_status
+ * clears those too.  The GPU context stays usable.
+ */
+int ap_selftest_wait_timeout(ap_kv_pool *pool, uint64_t limit_ns, int leave_counter, void *stream);
 
 /* ----------------------------------------------------------- diagnostics -- */
 
@@ -333,9 +359,9 @@ const char *ap_status_string(int status);
  * launching stream.  ap_profile_collect synchronises `stream`, adds up the
  * elapsed times per kernel since the last enable/collect, and clears the
  * records.  Index: 0 kv_append, 1 decode split-K (which also performs the LSE
- * merge), 2 unused, 3 prefill.
+ * merge), 2 prefill.
  */
-enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_MERGE = 2, AP_KERNEL_PREFILL = 3, AP_KERNEL_COUNT = 4 };
+enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_PREFILL = 2, AP_KERNEL_COUNT = 3 };
 typedef struct ap_kernel_times {
     double ms[AP_KERNEL_COUNT];
     int64_t launches[AP_KERNEL_COUNT];

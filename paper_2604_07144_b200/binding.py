@@ -39,6 +39,7 @@ EXPORTED_SYMBOLS = (
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
     "ap_static_workspace_bytes", "ap_attention_iteration_static",
+    "ap_kv_pool_set_wait_limit", "ap_selftest_wait_timeout",
 )
 
 
@@ -88,10 +89,10 @@ class PlanLayout(ctypes.Structure):
 
 
 class KernelTimes(ctypes.Structure):
-    _fields_ = [("ms", ctypes.c_double * 4), ("launches", ctypes.c_int64 * 4)]
+    _fields_ = [("ms", ctypes.c_double * 3), ("launches", ctypes.c_int64 * 3)]
 
 
-KERNEL_NAMES = ("kv_append", "decode_splitk", "lse_merge", "prefill")
+KERNEL_NAMES = ("kv_append", "decode_splitk", "prefill")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -135,6 +136,8 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_profile_collect": (ctypes.c_int, [vp, vp, ctypes.POINTER(KernelTimes)]),
         "ap_static_workspace_bytes": (sz, []),
         "ap_attention_iteration_static": (ctypes.c_int, [vp, vp, vp, vp, vp, vp]),
+        "ap_kv_pool_set_wait_limit": (ctypes.c_int, [vp, u64]),
+        "ap_selftest_wait_timeout": (ctypes.c_int, [vp, u64, ctypes.c_int, vp]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(lib, name)
@@ -382,6 +385,17 @@ def serving_iteration_host(pool: KVPool, q_lens, ctx_lens, block_tables, num_q_h
 
 def last_device_status(pool: KVPool, stream=None) -> int:
     return int(load().ap_last_device_status(pool.handle, _stream(stream)))
+
+
+def kv_pool_set_wait_limit(pool: KVPool, limit_ns: int) -> None:
+    """Bound (ns) of every wait inside the kernels launched for this pool from now on; 0 = default (2 s)."""
+    _check(load().ap_kv_pool_set_wait_limit(pool.handle, int(limit_ns)), "ap_kv_pool_set_wait_limit")
+
+
+def selftest_wait_timeout(pool: KVPool, limit_ns: int, leave_counter: bool = False, stream=None) -> None:
+    """Queues the one-warp kernel whose bounded wait always runs out (see ap_selftest_wait_timeout)."""
+    _check(load().ap_selftest_wait_timeout(pool.handle, int(limit_ns), int(bool(leave_counter)), _stream(stream)),
+           "ap_selftest_wait_timeout")
 
 
 # ------------------------------------------------------------ diagnostics --

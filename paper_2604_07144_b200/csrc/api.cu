@@ -223,7 +223,9 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
     if (desc->page_size != kPageSize) return AP_ERR_UNSUPPORTED;
     if (desc->head_dim != 64 && desc->head_dim != 128) return AP_ERR_UNSUPPORTED;
     if ((desc->k_base == nullptr) != (desc->v_base == nullptr)) return AP_ERR_INVALID_ARG;
-    if (((uintptr_t)desc->k_base | (uintptr_t)desc->v_base) & 1023u) return AP_ERR_INVALID_ARG;
+    // a tensor map's global address must be 16-byte aligned (the 1024-byte rule of the 128-byte
+    // swizzle concerns the shared-memory side, which the kernels align themselves)
+    if (((uintptr_t)desc->k_base | (uintptr_t)desc->v_base) & 15u) return AP_ERR_INVALID_ARG;
     // the tensor maps address 8-row groups with a 32-bit extent
     if ((int64_t)desc->num_pages * desc->num_kv_heads * 2 >= (int64_t)1 << 31) return AP_ERR_UNSUPPORTED;
 
@@ -279,6 +281,8 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
                 break;
             }
         }
+        rc = prepare_static_workspace(desc->device);
+        if (rc != AP_OK) break;
         rc = encode_pool_tensor_map(&p->k_map, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
         if (rc != AP_OK) break;
         rc = encode_pool_tensor_map(&p->v_map, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
@@ -835,6 +839,24 @@ int ap_last_device_status(ap_kv_pool *pool, void *stream) {
         }
     }
     return status;
+}
+
+int ap_kv_pool_set_wait_limit(ap_kv_pool *pool, uint64_t limit_ns) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    pool->wait_limit_ns = limit_ns ? limit_ns : kDefaultWaitLimitNs;
+    return AP_OK;
+}
+
+int ap_selftest_wait_timeout(ap_kv_pool *pool, uint64_t limit_ns, int leave_counter, void *stream) {
+    if (!pool || limit_ns == 0 || limit_ns > kDefaultWaitLimitNs) return AP_ERR_INVALID_ARG;
+    if (pool->desc.device < 0) return AP_ERR_CUDA;
+    DeviceGuard guard(pool->desc.device);
+    if (!guard.ok) return AP_ERR_CUDA;
+    if (launch_selftest_wait(pool, limit_ns, leave_counter != 0, (cudaStream_t)stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return AP_ERR_CUDA;
+    }
+    return AP_OK;
 }
 
 int ap_profile_enable(ap_kv_pool *pool, int on) {

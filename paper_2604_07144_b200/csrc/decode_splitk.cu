@@ -55,24 +55,6 @@ struct DecodeCfg {
     static_assert(kStages % 2 == 0, "consumer groups own alternate ring slots");
 };
 
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait: gives up after ~2 s (or when another warp has flagged abort).
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > 2000000000ull) return false;
-    }
-}
-
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
     uint32_t d;
     asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
@@ -184,7 +166,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                      const int32_t *__restrict__ cta_begin, const int32_t *__restrict__ bt_flat,
                      const MergeEntry *__restrict__ merges, float *o_part, float *lse_part,
                      __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out, int Hq, int Hkv, int G,
-                     int num_pages, float scale_log2, int *status) {
+                     int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns) {
     using Cfg = DecodeCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -258,7 +240,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                 const int ngroup = min(32, npages - p0);
                 for (int s0 = 0; s0 < ngroup; s0 += kPPS) {
                     const int n = min(kPPS, ngroup - s0);
-                    if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag)) {
+                    if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag, wait_limit_ns)) {
                         atomicCAS(status, 0, AP_ERR_TIMEOUT);
                         *abort_flag = 1;
                         return;
@@ -305,7 +287,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             const DecodeItem item = get_item(item_begin + pi);
             if (item.part_slot < 0) break;
             const MergeEntry me = merges[item.merge_index];
-            if (!wait_or_abort(&part_done[pi], 0, abort_flag)) {
+            if (!wait_or_abort(&part_done[pi], 0, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
@@ -343,7 +325,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         for (int it = item_begin; it < item_end; ++it) {
             const DecodeItem item = get_item(it);
             const int ti = it - item_begin, buf = ti & 1;
-            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti >> 1) & 1u, abort_flag)) {
+            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti >> 1) & 1u, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
@@ -416,7 +398,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             // arrive and signs it off.  A stage is refilled only after all eight warps are past it,
             // which keeps every waiter within one phase of each barrier (a parity wait is ambiguous
             // beyond that).
-            if (!wait_or_abort(&full[stage], phase, abort_flag)) {
+            if (!wait_or_abort(&full[stage], phase, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
@@ -508,7 +490,7 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         // ---- hand (m, l, O) to the combine warp through one of two shared-memory buffers and go on
         // with the next item; the buffer is reused two items later, once the combine warp has freed it
         const int ti = it - item_begin, buf = ti & 1;
-        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti >> 1) & 1u) ^ 1u, abort_flag)) {
+        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
             atomicCAS(status, 0, AP_ERR_TIMEOUT);
             *abort_flag = 1;
             return;
@@ -554,7 +536,7 @@ cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const v
         decode_splitk_kernel<D>, (unsigned)plan->info.decode_ctas, (unsigned)kDecodeThreads, (size_t)Cfg::kSmemBytes,
         stream, pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
         plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads,
-        plan->group, pool->desc.num_pages, scale_log2, pool->d_status);
+        plan->group, pool->desc.num_pages, scale_log2, pool->d_status, pool->wait_limit_ns);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -14,6 +14,7 @@
 namespace ap {
 
 constexpr int kPageSize = 16;
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;   // 2 s
 constexpr int kMaxMergeEntries = 4096;   // arrival counters kept per pool (the planner makes < 2 per CTA)
 
 // ---- device work lists (all int32, uploaded as one blob per plan) ---------
@@ -40,8 +41,9 @@ struct MergeEntry {
     int32_t part_count;
 };
 
-// One prefill work unit: 128 consecutive query rows of one sequence for one
-// q head, over all keys up to the last row's position.
+// One prefill work unit: 128 consecutive query rows of one sequence for two
+// q heads of the same kv head (or one, when the group has an odd head left),
+// over all keys up to the last row's position.
 struct PrefillTile {
     int32_t q_row0;      // global row of the tile's first query
     int32_t rows;        // valid rows in the tile (1..128)
@@ -88,6 +90,7 @@ struct ap_kv_pool {
     bool owns_planes = false;
     int sm_count = 0;
     int *d_status = nullptr;          // [0] status word, [1 ..] arrival counters of the merge entries
+    uint64_t wait_limit_ns = ap::kDefaultWaitLimitNs;   // bound of every wait inside a kernel
     CUtensorMap k_map{}, v_map{};
     // allocator
     std::vector<int32_t> free_list;     // pages handed out from the back
@@ -143,6 +146,8 @@ cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const vo
 // decode on `stream` and prefill on the pool's second stream, joined back into `stream`.
 cudaError_t launch_attention_kernels(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
                                      float *o_part, float *lse_part, cudaStream_t stream);
+// One warp waits on an mbarrier that nothing arrives on, with the given limit (see ap_selftest_wait_timeout).
+cudaError_t launch_selftest_wait(const ap_kv_pool *pool, uint64_t limit_ns, int leave_counter, cudaStream_t stream);
 // d_pairs: device [n_pairs][2] = (destination page, source page)
 cudaError_t launch_kv_copy_pages(const ap_kv_pool *dst_pool, const ap_kv_pool *src_pool, const int32_t *d_pairs,
                                  int n_pairs, cudaStream_t stream);
@@ -165,6 +170,9 @@ inline cudaError_t launch_overlapped(void (*kernel)(KArgs...), unsigned grid, un
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+
+// Per-device set-up of the library's fixed split-K scratch array (static_workspace.cu).
+int prepare_static_workspace(int device);
 
 // Decode kernel launch geometry (used by the planner to size the item lists).
 int decode_ctas_per_sm(int head_dim);

@@ -66,23 +66,6 @@ struct PrefillCfg {
     static constexpr uint32_t kColO = 256;    // + 128 * tile
 };
 
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > 2000000000ull) return false;
-    }
-}
-
 // three-input maximum (one instruction on sm_100)
 __device__ __forceinline__ float max3(float a, float b, float c) {
     float d;
@@ -146,7 +129,8 @@ __global__ void __launch_bounds__(kPrefillThreads, 1)
 prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                        const __grid_constant__ CUtensorMap v_map, const PrefillTile *__restrict__ tiles,
                        const int32_t *__restrict__ bt_flat, __nv_bfloat16 *__restrict__ out,
-                       float *__restrict__ lse_out, int Hq, int Hkv, int num_pages, float scale_log2, int *status) {
+                       float *__restrict__ lse_out, int Hq, int Hkv, int num_pages, float scale_log2, int *status,
+                       uint64_t wait_limit_ns) {
     using Cfg = PrefillCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -219,7 +203,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 const uint32_t ph = (uint32_t)(n / kKvSlots) & 1u;
                 const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
                 int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
-                if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag)) {
+                if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag, wait_limit_ns)) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                     break;
@@ -243,7 +227,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 const uint32_t leader = elect_one();
                 constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
                 constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
-                bool ok = wait_or_abort(q_full, 0, abort_flag);
+                bool ok = wait_or_abort(q_full, 0, abort_flag, wait_limit_ns);
                 // Descriptors are built once; per MMA only a constant is added to the address field
                 // (addresses are below 256 KB, so the 14-bit field cannot carry out).
                 // Q: [half][128 rows][64], 8-row groups 1024 B apart.  K: [16 groups of 8 keys][half][8][64].
@@ -277,7 +261,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         umma_ts_x4(leader, d, a + kq * 32, b0 + kq * 4 * kVStep, v_hi, kIdescPV,
                                    (first_step && kq == 0) ? 0u : 1u, 8u, kVStep);
                 };
-                if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag);
+                if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag, wait_limit_ns);
                 if (ok) {
                     tcgen05_fence_after();
                     for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);     // K_0 is ring entry 0, slot 0
@@ -285,14 +269,14 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
                     const int nv = kv_seq_v(j, n_steps), nk = kv_seq_k(j + 1);
-                    if (!wait_or_abort(&kv_full[nv % kKvSlots], (uint32_t)(nv / kKvSlots) & 1u, abort_flag)) { ok = false; break; }
+                    if (!wait_or_abort(&kv_full[nv % kKvSlots], (uint32_t)(nv / kKvSlots) & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                     for (int x = 0; x < n_tiles; ++x) {
-                        if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                        if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                         tcgen05_fence_after();
                         issue_pv(x, nv % kKvSlots, j == 0);
                         if (j + 1 < n_steps) {
                             if (x == 0 && !wait_or_abort(&kv_full[nk % kKvSlots], (uint32_t)(nk / kKvSlots) & 1u,
-                                                         abort_flag)) { ok = false; break; }
+                                                         abort_flag, wait_limit_ns)) { ok = false; break; }
                             issue_qk(x, nk % kKvSlots);                // overwrites S_x / P_x after the product above
                         } else {
                             umma_commit(leader, &o_done[x]);
@@ -323,7 +307,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             bool ok = true;
             for (int j = 0; j < n_steps; ++j) {
                 // S_x(j) complete; the same commit also covers O_x += P_x V of step j-1
-                if (!wait_or_abort(&s_full[x], (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+                if (!wait_or_abort(&s_full[x], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                 tcgen05_fence_after();
                 uint32_t sreg[4][32];
 #pragma unroll
@@ -391,7 +375,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                     // keys past the context hold no token: clear their V rows so 0 * garbage cannot
                     // poison O (tile A's group does it; tile B's product is issued after tile A's)
                     const int nv = kv_seq_v(j, n_steps), s = nv % kKvSlots;
-                    if (!wait_or_abort(&kv_full[s], (uint32_t)(nv / kKvSlots) & 1u, abort_flag)) { ok = false; break; }
+                    if (!wait_or_abort(&kv_full[s], (uint32_t)(nv / kKvSlots) & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                     uint8_t *v_tile = smem + Cfg::kOffK + s * Cfg::kKvTileBytes;
                     const int first = tile.ctx_len - tok0;           // first key of the step without a token
                     for (int idx = r; idx < (kTileN - first) * (D / 8); idx += 128) {
@@ -405,7 +389,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&p_full[x]);
             }
-            if (ok && wait_or_abort(&o_done[x], 0, abort_flag)) {
+            if (ok && wait_or_abort(&o_done[x], 0, abort_flag, wait_limit_ns)) {
                 tcgen05_fence_after();
                 const float inv = 1.f / l;
                 const bool valid = r < tile.rows;
@@ -461,7 +445,7 @@ cudaError_t launch_prefill_t(const ap_kv_pool *pool, const ap_plan *plan, const 
         prefill_tcgen05_kernel<D>, (unsigned)plan->info.prefill_tiles, (unsigned)kPrefillThreads,
         (size_t)Cfg::kSmemBytes, stream, q_map, pool->k_map, pool->v_map, plan->d_tiles, plan->d_bt_flat,
         (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, pool->desc.num_pages, scale_log2,
-        pool->d_status);
+        pool->d_status, pool->wait_limit_ns);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -1,7 +1,8 @@
 // Thin inline-PTX wrappers for sm_100a: mbarrier, bulk/tensor async copies
 // (TMA), ldmatrix / mma.sync, and tcgen05 (tensor memory + 5th-gen MMA).
-// Every wait is bounded: it gives up after a fixed number of polls and
-// reports failure to the caller, which records a status and unwinds.
+// Every wait goes through wait_or_abort: it is bounded by a time limit on the
+// global nanosecond timer (a kernel argument) and reports failure to the
+// caller, which records a status, raises the CTA's abort flag and unwinds.
 #pragma once
 
 #include <cuda.h>
@@ -61,15 +62,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Polls until the phase with the given parity has completed.  Returns false
-// after kWaitPolls unsuccessful polls (each poll may itself suspend the thread
-// for a hardware-defined interval), i.e. after seconds, never in normal
-// operation.
-constexpr uint32_t kWaitPolls = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitPolls; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Waits until the phase with the given parity has completed.  Gives up, returning false, once
+// `limit_ns` nanoseconds have passed or another warp of the CTA has raised the abort flag; the
+// clock is read only after the first unsuccessful poll, so a wait that succeeds at once costs one
+// try_wait.
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
+                                              uint64_t limit_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > limit_ns) return false;
+    }
 }
 
 // --------------------------------------------------------------------- TMA --

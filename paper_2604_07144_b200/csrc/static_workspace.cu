@@ -33,6 +33,19 @@ int static_workspace_address(int device, void **addr) {
 
 }  // namespace
 
+namespace ap {
+
+// Set-up step, run by ap_kv_pool_create with the pool's device current: looks the array's device
+// address up once per device.  The first lookup may make the runtime load this file's module (which
+// is when the array comes into being on that device), so it belongs where allocation is expected
+// and no stream is being captured, not in the serving loop.
+int prepare_static_workspace(int device) {
+    void *unused = nullptr;
+    return static_workspace_address(device, &unused);
+}
+
+}  // namespace ap
+
 extern "C" {
 
 size_t ap_static_workspace_bytes(void) { return kStaticWorkspaceBytes; }

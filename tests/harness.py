@@ -72,18 +72,58 @@ def oracle_pools(batch: W.Batch):
     return k, v
 
 
-def compare_outputs(out_bits: np.ndarray, lse: np.ndarray, ref_out: np.ndarray, ref_lse: np.ndarray, what=""):
+def out_tolerance(ref_out: np.ndarray) -> np.ndarray:
+    """Per-element bound on |bf16 output - fp64 oracle|.
+
+    1e-2 wherever |ref| < 2: there bf16 rounding of the result costs at most 2^-8 (half an ulp) and the
+    other error sources (weights P rounded to bf16 before the P V product: 2^-9 relative per weight;
+    ex2.approx; the cubic 2^x) stay well inside the rest.  A bf16 number with 2 <= |x| < 4 is only
+    known to 2^-7 (half an ulp: 7.8e-3) and with 4 <= |x| < 8 to 1.56e-2, so from |ref| = 2 on the format
+    alone eats the flat bound.  Such outputs need a softmax that is nearly one-hot on a large V entry
+    (short contexts, the first rows of a prompt; or a large explicit scale); for them the bound is what
+    the arithmetic gives: half an ulp of bf16 at ref plus 2^-8 |ref| for the rounded weights."""
+    a = np.abs(ref_out)
+    with np.errstate(divide="ignore"):
+        half_ulp = np.where(a > 0, 2.0 ** (np.floor(np.log2(np.maximum(a, 1e-300))) - 8), 0.0)
+    return np.where(a < 2.0, OUT_ATOL, half_ulp + a * 2.0 ** -8)
+
+
+def peaked_tolerance(ref_out: np.ndarray, abs_weighted: np.ndarray) -> np.ndarray:
+    """Bound for inputs that are NOT the N(0,1)-at-1/sqrt(d) case the flat 1e-2 is stated for (a large
+    explicit scale, keys that grow along the context): there the softmax is nearly one-hot, outputs are
+    close to copies of single V rows and a flat bound means little.  The arithmetic gives, per element,
+        |out - ref| <= 2^-9 * A  +  half an ulp of bf16 at ref  +  1e-3,
+    A = sum_j p_j |v_j| (the oracle's own result for |V|): every weight is rounded to bf16 before the P V
+    product (2^-9 relative each, the row sum is taken before rounding), the result is rounded to bf16
+    once, and 1e-3 covers ex2.approx, the cubic 2^x (7.7e-5 relative) and fp32 accumulation.  Tighter
+    than 1e-2 for most elements, looser only where |ref| or A is large."""
+    a = np.abs(ref_out)
+    half_ulp = np.where(a > 0, 2.0 ** (np.floor(np.log2(np.maximum(a, 1e-300))) - 8), 0.0)
+    return abs_weighted * 2.0 ** -9 + half_ulp + 1e-3
+
+
+def compare_outputs(out_bits: np.ndarray, lse: np.ndarray, ref_out: np.ndarray, ref_lse: np.ndarray, what="",
+                    abs_weighted=None):
     got = W.bf16_bits_to_f64(out_bits)
     assert np.isfinite(got).all(), f"{what}: non-finite output"
-    err = np.abs(got - ref_out).max() if got.size else 0.0
+    diff = np.abs(got - ref_out)
+    err = diff.max() if got.size else 0.0
     lerr = (np.abs(lse.astype(np.float64) - ref_lse) / np.maximum(np.abs(ref_lse), 1.0)).max() if lse.size else 0.0
-    assert err <= OUT_ATOL, f"{what}: out max abs err {err}"
+    if got.size:
+        tol = out_tolerance(ref_out) if abs_weighted is None else peaked_tolerance(ref_out, abs_weighted)
+        excess = diff - tol
+        i = np.unravel_index(np.argmax(excess), excess.shape)
+        assert excess[i] <= 0.0, (f"{what}: out error {diff[i]} at {i} (ref {ref_out[i]}, got {got[i]}) exceeds "
+                                  f"the bound {tol[i]}")
+        small = np.abs(ref_out) < 2.0
+        err = float(diff[small].max()) if small.any() else 0.0     # reported: the error where the flat 1e-2 applies
     assert lerr <= LSE_RTOL, f"{what}: lse rel err {lerr}"
     return float(err), float(lerr)
 
 
-def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None):
-    """Append + attention on the GPU against the oracle, every element."""
+def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None, peaked: bool = False):
+    """Append + attention on the GPU against the oracle, every element.  `peaked`: the inputs make the
+    softmax nearly one-hot, so the per-element bound of peaked_tolerance replaces the flat one."""
     run = GpuRun(batch, scale=scale, side_by_side=side_by_side)
     try:
         run.append()
@@ -96,8 +136,12 @@ def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None):
             return 0.0, 0.0
         ref_out, ref_lse = oracle.attention(k_ref, v_ref, batch.q_lens, batch.ctx_lens, batch.block_tables,
                                             batch.q, scale=scale)
+        abs_weighted = None
+        if peaked:       # the same attention over |V| (sign bit of every bf16 cleared): A = sum_j p_j |v_j|
+            abs_weighted, _ = oracle.attention(k_ref, v_ref & np.uint16(0x7FFF), batch.q_lens, batch.ctx_lens,
+                                               batch.block_tables, batch.q, scale=scale)
         return compare_outputs(to_bits(run.out)[:batch.n_new], run.lse.cpu().numpy()[:batch.n_new], ref_out,
-                               ref_lse, batch.name)
+                               ref_lse, batch.name, abs_weighted=abs_weighted)
     finally:
         run.close()
 

@@ -35,3 +35,27 @@ def test_status_strings():
     assert "block table" in binding.status_string(binding.AP_ERR_BAD_BLOCK_TABLE)
     assert binding.kv_pool_bytes(10, 8, 128) == 10 * 8 * 16 * 128 * 2
     assert binding.kv_pool_bytes(0, 8, 128) == 0
+
+
+def test_header_is_plain_c_and_struct_sizes_match_the_binding(tmp_path):
+    """include/ap_serving.h compiles as C99 on its own, and the structs the ctypes binding mirrors have
+    the sizes (and the enum the values) a C compiler gives them."""
+    import subprocess
+    src = tmp_path / "sizes.c"
+    src.write_text(
+        '#include "ap_serving.h"\n#include <stdio.h>\n'
+        "int main(void) {\n"
+        '  printf("%zu %zu %zu %zu %zu %zu %d %d %d\\n", sizeof(ap_pool_desc), sizeof(ap_batch_desc), sizeof(ap_plan_info),\n'
+        "         sizeof(ap_plan_prediction), sizeof(ap_plan_layout), sizeof(ap_kernel_times), (int)AP_KERNEL_COUNT,\n"
+        "         (int)AP_ERR_UNSUPPORTED, (int)AP_STATIC_WORKSPACE_BYTES);\n"
+        "  return 0;\n}\n")
+    exe = tmp_path / "sizes"
+    inc = os.path.join(ROOT, "include")
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", inc, "-fsyntax-only", "-x", "c",
+                           os.path.join(inc, "ap_serving.h")])
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", inc, str(src), "-o", str(exe)])
+    got = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    want = [ctypes.sizeof(binding.PoolDesc), ctypes.sizeof(binding.BatchDesc), ctypes.sizeof(binding.PlanInfo),
+            ctypes.sizeof(binding.PlanPrediction), ctypes.sizeof(binding.PlanLayout), ctypes.sizeof(binding.KernelTimes),
+            len(binding.KERNEL_NAMES), binding.AP_ERR_UNSUPPORTED, 4 << 20]
+    assert got == want

@@ -328,6 +328,104 @@ def test_prefill_chunk_shapes():
         check_batch_full(b)
 
 
+def test_decode_stream_cut_into_more_than_32_partials():
+    """One sequence, one kv head, 120 k tokens: the planner cuts the single (row, kv head) stream into
+    one item per SM, so the in-kernel LSE merge takes its chunked path (more partials than a warp has
+    lanes).  Every output against the oracle."""
+    b = decode_batch(107, (8, 1, 128), [120000], pool_factor=1.05)
+    run = GpuRun(b)
+    try:
+        ex = ap.plan_export(run.plan)
+        assert int(ex["merge_entries"][:, 3].max()) > 32, "the plan does not reach the chunked merge"
+    finally:
+        run.close()
+    err, lerr = check_batch_full(b)
+    print(f"148-way split: out err {err:.2e} lse err {lerr:.2e}")
+    # two such streams (G = 4 and G = 8 take different batch sizes in the merge's fetch loop)
+    check_batch_full(decode_batch(108, (8, 2, 128), [70000], pool_factor=1.05))
+    check_batch_full(decode_batch(109, (2, 1, 64), [90000], pool_factor=1.05))
+
+
+def test_decode_more_items_per_cta_than_the_shared_memory_list_holds():
+    """1500 short decode rows x 8 kv heads = 12 000 items, ~81 per CTA: past the 64 item descriptors a
+    CTA keeps in shared memory, so the rest come from global memory.  Every output against the oracle."""
+    rng = np.random.default_rng(11)
+    b = decode_batch(110, W.SHAPE_8B, rng.integers(1, 49, size=1500))
+    run = GpuRun(b)
+    try:
+        ex = ap.plan_export(run.plan)
+        assert int(np.diff(ex["cta_begin"]).max()) > 64, "no CTA holds more than 64 items"
+    finally:
+        run.close()
+    err, lerr = check_batch_full(b)
+    print(f"12000 items: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def _prefill_rescales(batch, scale, head=0, seq=0):
+    """How often the prefill kernel's rule "rescale O when some row of a 32-row group sees its running
+    maximum rise by more than 8 (log2 units) after the first step" fires for one (sequence, q head),
+    worked out from the inputs in fp64 (test-side bookkeeping of which inputs reach that path)."""
+    from harness import oracle_pools
+    k_ref, _ = oracle_pools(batch)
+    hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
+    g = head // (hq // hkv)
+    ql, cl = int(batch.q_lens[seq]), int(batch.ctx_lens[seq])
+    pages = batch.block_tables[seq, :(cl + 15) // 16]
+    k = W.bf16_bits_to_f64(k_ref[pages, g]).reshape(-1, d)[:cl]
+    r0 = int(batch.q_indptr[seq])
+    q = W.bf16_bits_to_f64(batch.q[r0:r0 + ql, head])
+    s = (q @ k.T) * scale * np.log2(np.e)
+    pos = cl - ql + np.arange(ql)
+    s[np.arange(cl)[None, :] > pos[:, None]] = -np.inf
+    fired = 0
+    for t0 in range(0, ql, 128):
+        rows = s[t0:t0 + 128]
+        n_steps = (int(pos[min(t0 + 127, ql - 1)]) + 1 + 127) // 128
+        for w0 in range(0, rows.shape[0], 32):
+            blk = rows[w0:w0 + 32]
+            m_used = np.full(blk.shape[0], -np.inf)
+            for j in range(n_steps):
+                mx = blk[:, j * 128:(j + 1) * 128].max(axis=1)
+                m_new = np.maximum(m_used, mx)
+                with np.errstate(invalid="ignore"):
+                    moved = (m_new - m_used) > 8.0
+                if moved.any():
+                    m_used = m_new
+                    fired += j > 0
+    return fired
+
+
+@pytest.mark.parametrize("shape,scale", [((4, 2, 64), 1.0), ((4, 2, 64), 0.5), (W.SHAPE_8B, 0.5), ((6, 2, 128), 0.7)],
+                         ids=["d64_scale1", "d64_scale0.5", "8B_scale0.5", "G3_scale0.7"])
+def test_prefill_explicit_scale_rescales_the_accumulator(shape, scale):
+    """Prefill with an explicit softmax scale large enough that row maxima keep climbing after the
+    first key step, so O is rescaled in tensor memory (the kernel's rare path); against the oracle at
+    the same scale, same tolerances."""
+    b = W._assemble("prefill_scale", shape, W.make_rng(320), np.array([384, 1, 200], np.int32),
+                    np.array([1400, 300, 200], np.int32), 1.3)
+    assert _prefill_rescales(b, scale) > 0, "these inputs never move the running maximum by more than 8"
+    err, lerr = check_batch_full(b, scale=scale, peaked=True)
+    print(f"prefill scale {scale}: out err {err:.2e} lse err {lerr:.2e}")
+
+
+def test_prefill_keys_growing_along_the_context():
+    """Default scale, but K grows with the position (norm x1 ... x4 over the context), so every row's
+    maximum rises step after step and the O rescale fires at the standard 1/sqrt(d)."""
+    b = W._assemble("prefill_growing_k", W.SHAPE_8B, W.make_rng(321), np.array([256, 1], np.int32),
+                    np.array([2304, 500], np.int32), 1.3)
+    cl, ql = int(b.ctx_lens[0]), int(b.q_lens[0])
+    grow = lambda j: 1.0 + 3.0 * j / cl
+    for j in range(cl - ql):                           # cached keys, through the block table
+        page, slot = int(b.block_tables[0, j // 16]), j % 16
+        b.k_pool[page, :, slot] = W.f32_to_bf16_bits((W.bf16_bits_to_f64(b.k_pool[page, :, slot]) * grow(j)).astype(np.float32))
+    for t in range(ql):                                # this iteration's keys
+        b.k_new[t] = W.f32_to_bf16_bits((W.bf16_bits_to_f64(b.k_new[t]) * grow(cl - ql + t)).astype(np.float32))
+    b.q[:ql] = W.f32_to_bf16_bits((W.bf16_bits_to_f64(b.q[:ql]) * 1.5).astype(np.float32))
+    assert _prefill_rescales(b, 1.0 / np.sqrt(b.head_dim)) > 0
+    err, lerr = check_batch_full(b, peaked=True)
+    print(f"prefill growing K: out err {err:.2e} lse err {lerr:.2e}")
+
+
 def test_prefill_long_prefix_and_maximum_chunk():
     """The largest prefill work the configurations allow: a chunk deep inside a long context (485 key
     steps per unit, the K/V ring wraps ~190 times) and a whole 8192-token prompt in one iteration (the
@@ -357,83 +455,136 @@ def test_workspace_too_small_is_reported():
     run.close()
 
 
-def test_config2_full_size_sampled():
-    err, lerr = check_batch_sampled(W.config2(), n_samples=256)
-    print(f"config2: out err {err:.2e} lse err {lerr:.2e}")
+@pytest.mark.parametrize("config", [2, 3, 4])
+def test_full_size_configs_every_output(config):
+    """Configurations 2, 3 and 4 at full size, in the launch configuration the benchmark times (the
+    planner's own dispatch mode): whole-pool bit comparison after the append and EVERY attention output
+    and lse against the oracle."""
+    batch = {2: W.config2, 3: W.config3, 4: W.config4}[config]()
+    err, lerr = check_batch_full(batch)
+    print(f"config{config}: every output, out err {err:.2e} lse err {lerr:.2e}")
 
 
-def test_config3_full_size_sampled():
-    err, lerr = check_batch_sampled(W.config3(), n_samples=256)
-    print(f"config3: out err {err:.2e} lse err {lerr:.2e}")
+def test_config3_sequential_dispatch_every_output():
+    """Config 3 once more with decode and prefill one after the other (the mode the per-kernel
+    roofline figures are taken in)."""
+    err, lerr = check_batch_full(W.config3(), side_by_side=0)
+    print(f"config3 sequential: out err {err:.2e} lse err {lerr:.2e}")
 
 
-def test_config4_full_size_sampled():
-    err, lerr = check_batch_sampled(W.config4(), n_samples=48)
-    print(f"config4: out err {err:.2e} lse err {lerr:.2e}")
-
-
-def test_host_buffer_iteration_matches_device_path():
+def test_host_buffer_iteration_against_the_oracle():
+    """ap_serving_iteration_host (plan, copies in, append, attention, copies out, one sync) on a mixed
+    batch with cut decode streams, from pinned host buffers: pool bit-exact and every output against
+    the oracle; the device-buffer path on a second pool must give the same bits."""
     import torch
-    b = W.random_ragged(501, shape=W.SHAPE_8B, batch=6, max_ctx=500, max_q=1)
-    b.q_lens[:] = 1
-    b = decode_batch(502, W.SHAPE_8B, [77, 500, 1300, 16])
+    import oracle
+    from harness import compare_outputs, oracle_pools
+    b = W._assemble("host_buffers", W.SHAPE_8B, W.make_rng(502), np.array([1, 1, 150, 1, 1], np.int32),
+                    np.array([77, 9000, 400, 1300, 16], np.int32), 1.3)
+    k_ref, v_ref = oracle_pools(b)
+    ref_out, ref_lse = oracle.attention(k_ref, v_ref, b.q_lens, b.ctx_lens, b.block_tables, b.q)
     run = GpuRun(b)
-    run.append(); run.attend()
-    assert run.status() == 0
-    ref_out, ref_lse = to_bits(run.out)[:b.n_new].copy(), run.lse.cpu().numpy()[:b.n_new].copy()
-    ref_k = to_bits(run.k_pool).copy()
-    run.close()
-    run = GpuRun(b)                                  # fresh pool (pre-append state)
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
-    q, kn, vn = pin(b.q), pin(b.k_new), pin(b.v_new)
-    out = torch.empty((b.n_new, b.num_q_heads, b.head_dim), dtype=torch.int16).pin_memory()
-    lse = torch.empty((b.n_new, b.num_q_heads), dtype=torch.float32).pin_memory()
-    ap.serving_iteration_host(run.pool, b.q_lens, b.ctx_lens, b.block_tables, b.num_q_heads, q, kn, vn, out, lse)
-    assert np.array_equal(out.numpy().view(np.uint16), ref_out)
-    assert np.array_equal(lse.numpy(), ref_lse)
-    assert np.array_equal(to_bits(run.k_pool), ref_k)
-    run.close()
+    try:
+        assert run.info["merge_entries"] > 0
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
+        q, kn, vn = pin(b.q), pin(b.k_new), pin(b.v_new)
+        out = torch.empty((b.n_new, b.num_q_heads, b.head_dim), dtype=torch.int16).pin_memory()
+        lse = torch.empty((b.n_new, b.num_q_heads), dtype=torch.float32).pin_memory()
+        for _ in range(2):                               # the second call reuses the pool's staging buffers
+            out.fill_(0x7FC1); lse.fill_(float("nan"))
+            ap.serving_iteration_host(run.pool, b.q_lens, b.ctx_lens, b.block_tables, b.num_q_heads, q, kn, vn, out, lse)
+            compare_outputs(out.numpy().view(np.uint16), lse.numpy(), ref_out, ref_lse, "host buffers")
+        assert np.array_equal(to_bits(run.k_pool), k_ref) and np.array_equal(to_bits(run.v_pool), v_ref)
+        host_out, host_lse = out.numpy().view(np.uint16).copy(), lse.numpy().copy()
+    finally:
+        run.close()
+    run = GpuRun(b)
+    try:
+        run.append(); run.attend()
+        assert run.status() == 0
+        assert np.array_equal(to_bits(run.out)[:b.n_new], host_out)
+        assert np.array_equal(run.lse.cpu().numpy()[:b.n_new], host_lse)
+    finally:
+        run.close()
+
+
+def _trace_full_check_iterations(budget, chunk, iterations=200):
+    """Iterations of the trace whose every output is compared: the one with the largest plan (most
+    decode work items), the one where a decode CTA's item list is longest, and the one with the most
+    new tokens; found by a dry run of the scheduler on a host-only pool (which plans like a 148-SM GPU)."""
+    from paper_2604_07144_b200 import binding as B_
+    reqs = W.trace_arrivals(W.SEED_BASE + 5, iterations)
+    alloc = W.FreeListAllocator(1 << 22)
+    hq, hkv, d = W.SHAPE_8B
+    pool = ap.kv_pool_create(1 << 22, hkv, d, device=-1)
+    best_items, best_new, best_list = (-1, -1), (-1, -1), (-1, -1)
+    for it in W.fcfs_trace(reqs, alloc.alloc, alloc.free, iterations=iterations, token_budget=budget, chunk=chunk):
+        if int(it.q_lens.sum()) == 0:
+            continue
+        plan = ap.plan_create(pool, it.q_lens, it.ctx_lens, it.block_tables, hq)
+        ex = ap.plan_export(plan)
+        ap.plan_destroy(plan)
+        per_cta = int(np.diff(ex["cta_begin"]).max()) if len(ex["cta_begin"]) > 1 else 0
+        best_items = max(best_items, (ex["info"]["decode_items"], it.index))
+        best_list = max(best_list, (per_cta, it.index))
+        best_new = max(best_new, (int(it.q_lens.sum()), it.index))
+    ap.kv_pool_destroy(pool)
+    return {best_items[1], best_new[1], best_list[1]}, best_list[0]
 
 
 @pytest.mark.parametrize("budget,chunk", [(8192, 512), (2048, 256)], ids=["budget8192_chunk512", "budget2048_chunk256"])
 def test_config5_trace_parity(budget, chunk):
-    """Workload-shift trace (shortened to 80 iterations, across the rate switch at 50), under the
-    configuration's scheduler and under a second fixed policy: pages come from the library's
-    allocator and are freed per request; the pool must match the oracle's bit for bit at the end,
-    and sampled attention outputs every iteration must be in tolerance."""
+    """The whole 200-iteration workload-shift trace (both low-rate and both high-rate phases), under
+    the configuration's scheduler and under a second fixed policy: pages come from the library's
+    allocator and are freed per request; the pool must match the oracle's bit for bit at the end;
+    every iteration is compared on sampled outputs, and the iterations with the largest plan and with
+    the most new tokens on every output."""
     import oracle
     from harness import compare_outputs
     from paper_2604_07144_b200.trace_runner import TraceRun
-    run = TraceRun(iterations=80, token_budget=budget, chunk=chunk)
+    full_iters, longest_list = _trace_full_check_iterations(budget, chunk)
+    if budget == 8192:
+        assert longest_list > 64      # the trace's largest plan overflows a CTA's shared-memory item list
+    run = TraceRun(iterations=200, token_budget=budget, chunk=chunk)
     hq, hkv, d = run.shape
     k_ref = np.full((run.num_pages, hkv, 16, d), W.CANARY, np.uint16)
     v_ref = k_ref.copy()
     rng = np.random.default_rng(55)
-    seen_prefill = seen_decode = checked = 0
+    seen_prefill = seen_decode = checked = full_checked = 0
+    last_index = -1
     worst = (0.0, 0.0)
     try:
         for st in run.steps():
+            last_index = st.index
             if st.q is None:
                 continue
             assert oracle.kv_append(k_ref, v_ref, st.q_lens, st.ctx_lens, st.block_tables, st.k_new, st.v_new) == 0
             seen_prefill += st.n_prefill
             seen_decode += st.n_decode
-            n = 12
-            seq = rng.integers(0, len(st.q_lens), size=n)
-            tok = np.array([rng.integers(0, st.q_lens[s]) for s in seq], dtype=np.int32)
-            head = rng.integers(0, hq, size=n).astype(np.int32)
-            ref_out, ref_lse = oracle.attention_samples(k_ref, v_ref, st.q_lens, st.ctx_lens, st.block_tables, st.q,
-                                                        seq, tok, head)
-            rows = np.concatenate([[0], np.cumsum(st.q_lens)])[seq] + tok
-            out = to_bits(st.out)[rows, head]
-            lse = st.lse.cpu().numpy()[rows, head]
-            e = compare_outputs(out, lse, ref_out, ref_lse, f"trace iteration {st.index}")
+            if st.index in full_iters:
+                ref_out, ref_lse = oracle.attention(k_ref, v_ref, st.q_lens, st.ctx_lens, st.block_tables, st.q)
+                e = compare_outputs(to_bits(st.out), st.lse.cpu().numpy(), ref_out, ref_lse,
+                                    f"trace iteration {st.index}, every output")
+                full_checked += 1
+                checked += ref_lse.size
+            else:
+                n = 12
+                seq = rng.integers(0, len(st.q_lens), size=n)
+                tok = np.array([rng.integers(0, st.q_lens[s]) for s in seq], dtype=np.int32)
+                head = rng.integers(0, hq, size=n).astype(np.int32)
+                ref_out, ref_lse = oracle.attention_samples(k_ref, v_ref, st.q_lens, st.ctx_lens, st.block_tables,
+                                                            st.q, seq, tok, head)
+                rows = np.concatenate([[0], np.cumsum(st.q_lens)])[seq] + tok
+                e = compare_outputs(to_bits(st.out)[rows, head], st.lse.cpu().numpy()[rows, head], ref_out, ref_lse,
+                                    f"trace iteration {st.index}")
+                checked += n
             worst = (max(worst[0], e[0]), max(worst[1], e[1]))
-            checked += n
-        assert seen_prefill > 0 and seen_decode > 0 and checked > 500
+        assert last_index == 199 and full_checked == len(full_iters)
+        assert seen_prefill > 0 and seen_decode > 0 and checked > 2000
         assert np.array_equal(to_bits(run.k_pool), k_ref), "K plane differs after the trace"
         assert np.array_equal(to_bits(run.v_pool), v_ref), "V plane differs after the trace"
-        print(f"config5 (80 iterations): {checked} sampled outputs, out err {worst[0]:.2e} lse err {worst[1]:.2e}")
+        print(f"config5 (200 iterations, {sorted(full_iters)} in full): {checked} outputs, out err {worst[0]:.2e} "
+              f"lse err {worst[1]:.2e}")
     finally:
         run.close()
 
@@ -445,3 +596,38 @@ def test_prefill_head_ratios(shape):
     b = W._assemble("prefill_heads", shape, W.make_rng(600), np.array([150, 1, 70], np.int32),
                     np.array([333, 90, 70], np.int32), 1.3)
     check_batch_full(b)
+
+
+def test_bounded_wait_times_out_and_the_pool_recovers():
+    """The kernels' failure path in the only form that harms nothing: a one-warp kernel waits, through
+    the bounded-wait routine the attention kernels use, on a barrier nothing arrives on.  It must end by
+    itself, leave AP_ERR_TIMEOUT in the pool's status word (returned once, then cleared) together with a
+    raised split-K arrival counter (cleared with it), and the next ordinary iteration on the same pool,
+    one with cut streams, must be right."""
+    import time
+    import torch
+    import oracle
+    from harness import compare_outputs, oracle_pools
+    b = decode_batch(120, W.SHAPE_8B, [20000, 9001, 333])
+    run = GpuRun(b)
+    try:
+        assert run.info["merge_entries"] > 0
+        with pytest.raises(ap.ApError):
+            ap.selftest_wait_timeout(run.pool, 0)                    # a limit is required
+        t0 = time.perf_counter()
+        ap.selftest_wait_timeout(run.pool, 1_000_000, leave_counter=True)       # 1 ms
+        assert run.status() == B.AP_ERR_TIMEOUT
+        assert time.perf_counter() - t0 < 1.0
+        assert run.status() == 0                                         # reported once
+        ap.kv_pool_set_wait_limit(run.pool, 500_000_000)                 # a pool setting; kernels take it as an argument
+        run.append(); run.attend()
+        assert run.status() == 0
+        k_ref, v_ref = oracle_pools(b)
+        ref_out, ref_lse = oracle.attention(k_ref, v_ref, b.q_lens, b.ctx_lens, b.block_tables, b.q)
+        compare_outputs(to_bits(run.out)[:b.n_new], run.lse.cpu().numpy()[:b.n_new], ref_out, ref_lse, "after a timeout")
+        ap.kv_pool_set_wait_limit(run.pool, 0)
+        run.attend()
+        assert run.status() == 0
+        assert torch.cuda.is_available()
+    finally:
+        run.close()

@@ -10,8 +10,10 @@ that keeps the split-K partials in a fixed 4 MiB array of its own.
 This test drives that variant through the C ABI and requires the same output
 as the ordinary entry point on two calls in a row (the second call sees the
 scratch exactly as the first one left it, and a different batch in between
-makes sure stale partials are never picked up).  It lives in the file pytest
-collects last, so a failure here cannot hide the result of any other test.
+makes sure stale partials are never picked up); both are also held against
+the CPU oracle, and the amount of free device memory must not move across the
+calls.  It lives in the file pytest collects last, so a failure here cannot
+hide the result of any other test.
 """
 import numpy as np
 import pytest
@@ -20,7 +22,7 @@ import paper_2604_07144_b200 as ap
 from paper_2604_07144_b200 import binding as B
 from paper_2604_07144_b200 import workloads as W
 
-from harness import GpuRun, LSE_RTOL, OUT_ATOL, to_bits
+from harness import GpuRun, LSE_RTOL, OUT_ATOL, oracle_pools, to_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -49,6 +51,13 @@ def _static(run):
     return W.bf16_bits_to_f64(to_bits(run.out)[:n]), run.lse.cpu().numpy()[:n].astype(np.float64)
 
 
+def _oracle(batch):
+    """The CPU oracle's result for the batch (append, then attention of every new token)."""
+    import oracle
+    k_ref, v_ref = oracle_pools(batch)
+    return oracle.attention(k_ref, v_ref, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.q)
+
+
 def _same(got, ref):
     out, lse = got
     ref_out, ref_lse = ref
@@ -66,10 +75,26 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
         assert a.info["merge_entries"] > 0 and b.info["merge_entries"] > 0
         assert 0 < a.workspace_bytes <= ap.static_workspace_bytes()
         ref_a, ref_b = _reference(a), _reference(b)
-        _same(_static(a), ref_a)          # first call (does the one-time address lookup)
-        _same(_static(a), ref_a)          # second call in a row, scratch holds the first call's partials
-        _same(_static(b), ref_b)          # another batch over the same scratch
+        ora_a, ora_b = _oracle(a.batch), _oracle(b.batch)
+        _same(ref_a, ora_a)
+        _same(ref_b, ora_b)
+        first = _static(a)                # first call on this pool
+        _same(first, ref_a)
+        _same(first, ora_a)
+        import torch
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        second = _static(a)               # second call in a row, scratch holds the first call's partials
+        _same(second, ref_a)
+        _same(second, ora_a)
+        other = _static(b)                # another batch over the same scratch
+        _same(other, ref_b)
+        _same(other, ora_b)
         _same(_static(a), ref_a)
+        torch.cuda.synchronize()
+        # nothing was allocated on the device by any of those calls (the comparisons above only
+        # made host copies; torch's caching allocator serves them from blocks it already holds)
+        assert torch.cuda.mem_get_info()[0] >= free_before
     finally:
         a.close()
         b.close()
@@ -85,7 +110,10 @@ def test_static_workspace_with_a_mixed_plan_run_side_by_side():
     try:
         assert run.info["side_by_side"] == 1 and run.info["merge_entries"] > 0
         ref = _reference(run)
-        _same(_static(run), ref)
+        ora = _oracle(batch)
+        got = _static(run)
+        _same(got, ref)
+        _same(got, ora)
         _same(_static(run), ref)
     finally:
         run.close()
