@@ -14,11 +14,16 @@
 //               of the second product, rescale O in TMEM when the running max has
 //               moved enough, and write the normalised output at the end
 //   warp 8      producer: Q tiles once, then K and V tiles into one 5-slot ring
-//   warp 9      MMA issuer (converged warp, one elected lane issues): S_x = Q_x K^T, O_x += P_x V for x = A, B in turn, so the
-//               tensor pipe works on one tile while the other tile's softmax runs
-//   warps 10-11 idle (they only complete the third warpgroup for the register split)
+//   warps 9, 10 MMA issuers, one per tile (converged warp, one elected lane issues): S = Q_x K^T, O_x += P_x V;
+//               the tensor pipe works on one tile while the other tile's softmax runs
+//   warp 11     idle (it only completes the third warpgroup for the register split)
 //
-// TMEM columns: S_A/P_A 0-127, S_B/P_B 128-255, O_A 256-.., O_B 384-.. (512 allocated).
+// TMEM columns: S 0-127 (ONE score region that tiles A and B use in turn), P_A 128-191, P_B 192-255,
+// O_A 256-.., O_B 384-.. (512 allocated).  A softmax group copies its S tile into registers at once and
+// hands the region back (s_out), and P has columns of its own, so the next scores of a tile,
+// S_x(j+1), do not have to wait for O_x += P_x(j) V: they are issued ahead of it.  The order on the
+// tensor pipe is  S_A(j+1), P_A(j) V, S_B(j+1), P_B(j) V;  per tile only softmax(j) -> softmax(j+1)
+// remains as a chain, instead of softmax -> P V -> Q K^T -> softmax.
 // Registers: the block is launched with 168 registers per thread; the third
 // warpgroup drops to 72 and the two softmax groups raise themselves to 216
 // (128 * 72 + 256 * 216 = 384 * 168), so a whole S row fits in registers.
@@ -62,7 +67,8 @@ struct PrefillCfg {
     static constexpr int kOffBar = kOffK + kKvSlots * kKvTileBytes;
     static constexpr int kSmemBytes = 1024 + kOffBar + 256;
     static constexpr uint32_t kTmemCols = 512;
-    static constexpr uint32_t kColS = 0;      // + 128 * tile
+    static constexpr uint32_t kColS = 0;      // shared by both tiles
+    static constexpr uint32_t kColP = 128;    // + 64 * tile (bf16 pairs)
     static constexpr uint32_t kColO = 256;    // + 128 * tile
 };
 
@@ -140,8 +146,9 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
     uint64_t *kv_empty = kv_full + kKvSlots;     // [kKvSlots]
     uint64_t *s_full = kv_empty + kKvSlots;      // [2] per tile
     uint64_t *p_full = s_full + 2;               // [2]
-    uint64_t *o_done = p_full + 2;               // [2]
-    uint32_t *tmem_slot = (uint32_t *)(o_done + 2);
+    uint64_t *pv_done = p_full + 2;              // [2] O_x += P_x V of a step has completed
+    uint64_t *s_out = pv_done + 2;               // [2] tile x's scores have been copied out of the shared region
+    uint32_t *tmem_slot = (uint32_t *)(s_out + 2);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -155,12 +162,13 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
         mbar_init(q_full, 1);
         for (int s = 0; s < kKvSlots; ++s) {
             mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
+            mbar_init(&kv_empty[s], n_tiles);    // one commit per issuing warp
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&s_full[x], 1);
             mbar_init(&p_full[x], 4);            // one arrival per softmax warp
-            mbar_init(&o_done[x], 1);
+            mbar_init(&pv_done[x], 1);
+            mbar_init(&s_out[x], 4);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -220,10 +228,15 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                                 is_k ? &k_map : &v_map, &kv_full[s], 0, 0, 0, group);
                 }
             }
-        } else if (warp == kMmaWarp) {
-            // ------------------------------------------------ MMA issuer --
-            // The warp runs this block converged; `leader` selects the lane that issues.
+        } else if (warp == kMmaWarp || (warp == kMmaWarp + 1 && n_tiles == 2)) {
+            // ----------------------------------------------- MMA issuers --
+            // One issuing warp per tile (warp 9: tile A, warp 10: tile B), so that one tile's wait for
+            // its P does not hold up the other tile's instructions.  Each warp runs this block
+            // converged; `leader` selects the lane that issues.  The two meet only in barriers: the
+            // score region passes from one tile to the other through s_free, and a K/V slot is
+            // released when both have committed their last product on it.
             {
+                const int x = warp - kMmaWarp;
                 const uint32_t leader = elect_one();
                 constexpr uint32_t kIdescQK = instr_desc(kTileM, kTileN, false);
                 constexpr uint32_t kIdescPV = instr_desc(kTileM, D, true);
@@ -232,59 +245,70 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 // (addresses are below 256 KB, so the 14-bit field cannot carry out).
                 // Q: [half][128 rows][64], 8-row groups 1024 B apart.  K: [16 groups of 8 keys][half][8][64].
                 // V (MN-major): 64-column halves 1024 B apart (LBO), 8-key groups 1024 * halves apart (SBO).
-                const uint64_t q_desc0 = smem_desc(smem_u32(smem + Cfg::kOffQ), 16, 1024);
+                const uint64_t q_desc0 = smem_desc(smem_u32(smem + Cfg::kOffQ + x * Cfg::kQBytes), 16, 1024);
                 const uint64_t k_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 16, 1024 * Cfg::kHalves);
                 const uint64_t v_desc0 = smem_desc(smem_u32(smem + Cfg::kOffK), 1024, 1024 * Cfg::kHalves);
                 const uint32_t q_lo = (uint32_t)q_desc0, q_hi = (uint32_t)(q_desc0 >> 32);
                 const uint32_t k_lo = (uint32_t)k_desc0, k_hi = (uint32_t)(k_desc0 >> 32);
                 const uint32_t v_lo = (uint32_t)v_desc0, v_hi = (uint32_t)(v_desc0 >> 32);
-                // S_x = Q_x K^T with K in ring slot `slot`
-                auto issue_qk = [&](int x, int slot) {
-                    const uint32_t a0 = q_lo + (uint32_t)((x * Cfg::kQBytes) >> 4);
+                const uint32_t t_s = tmem + Cfg::kColS, t_p = tmem + Cfg::kColP + x * 64, t_o = tmem + Cfg::kColO + x * 128;
+                // S = Q_x K^T with K in ring slot `slot`, into the shared score region
+                auto issue_qk = [&](int slot) {
                     const uint32_t b0 = k_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
-                    const uint32_t d = tmem + Cfg::kColS + x * 128;
                     // 16 elements of d per MMA: 32 bytes further inside the 64-element half, next half every four
 #pragma unroll
                     for (int kh = 0; kh < D / 64; ++kh)
-                        umma_ss_x4(leader, d, a0 + (uint32_t)((kh * (kTileM * 128)) >> 4), q_hi,
+                        umma_ss_x4(leader, t_s, q_lo + (uint32_t)((kh * (kTileM * 128)) >> 4), q_hi,
                                    b0 + (uint32_t)((kh * 1024) >> 4), k_hi, kIdescQK, kh > 0 ? 1u : 0u, 32u >> 4, 32u >> 4);
                     umma_commit(leader, &s_full[x]);
+                    umma_commit(leader, &kv_empty[slot]);
                 };
-                // O_x += P_x V with V in ring slot `slot`.  P: bf16 pairs in the first 64 columns of S_x
+                // O_x += P_x V with V in ring slot `slot`.  P_x: bf16 pairs in 64 columns of its own
                 // (A operand from TMEM, 8 columns per 16 keys); 16 keys of V = 2 groups of 8.
-                auto issue_pv = [&](int x, int slot, bool first_step) {
+                auto issue_pv = [&](int slot, bool first_step) {
                     const uint32_t b0 = v_lo + (uint32_t)((slot * Cfg::kKvTileBytes) >> 4);
-                    const uint32_t d = tmem + Cfg::kColO + x * 128, a = tmem + Cfg::kColS + x * 128;
                     constexpr uint32_t kVStep = (uint32_t)((2 * 1024 * Cfg::kHalves) >> 4);   // 16 keys of V
 #pragma unroll
                     for (int kq = 0; kq < kTileN / 64; ++kq)
-                        umma_ts_x4(leader, d, a + kq * 32, b0 + kq * 4 * kVStep, v_hi, kIdescPV,
+                        umma_ts_x4(leader, t_o, t_p + kq * 32, b0 + kq * 4 * kVStep, v_hi, kIdescPV,
                                    (first_step && kq == 0) ? 0u : 1u, 8u, kVStep);
+                    umma_commit(leader, &pv_done[x]);
+                    umma_commit(leader, &kv_empty[slot]);
+                };
+                // The score region is used by one tile after the other: use number u = step * tiles + x
+                // may be issued once the softmax group of use u - 1 has copied its scores out.
+                // S_x(step) may be issued once the scores written before it have been copied out: with two
+                // tiles, S_B(step - 1) before S_A(step) and S_A(step) before S_B(step); with one, S_A(step - 1).
+                // Each of the two barriers has one waiter that follows it phase by phase (a parity wait can
+                // only tell the current phase from the one before).
+                auto wait_s_free = [&](int step) {
+                    if (n_tiles == 2 && x == 1) return wait_or_abort(&s_out[0], (uint32_t)step & 1u, abort_flag, wait_limit_ns);
+                    if (step == 0) return true;
+                    return wait_or_abort(&s_out[n_tiles - 1], (uint32_t)(step - 1) & 1u, abort_flag, wait_limit_ns);
                 };
                 if (ok) ok = wait_or_abort(&kv_full[0], 0, abort_flag, wait_limit_ns);
+                if (ok) ok = wait_s_free(0);
                 if (ok) {
                     tcgen05_fence_after();
-                    for (int x = 0; x < n_tiles; ++x) issue_qk(x, 0);     // K_0 is ring entry 0, slot 0
-                    umma_commit(leader, &kv_empty[0]);
+                    issue_qk(0);                                        // K_0 is ring entry 0, slot 0
                 }
                 for (int j = 0; ok && j < n_steps; ++j) {
                     const int nv = kv_seq_v(j, n_steps), nk = kv_seq_k(j + 1);
-                    if (!wait_or_abort(&kv_full[nv % kKvSlots], (uint32_t)(nv / kKvSlots) & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
-                    for (int x = 0; x < n_tiles; ++x) {
-                        if (!wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
+                    if (j + 1 < n_steps) {
+                        // the next scores of the tile go ahead of this step's P V
+                        if (!wait_or_abort(&kv_full[nk % kKvSlots], (uint32_t)(nk / kKvSlots) & 1u, abort_flag,
+                                           wait_limit_ns) || !wait_s_free(j + 1)) { ok = false; break; }
                         tcgen05_fence_after();
-                        issue_pv(x, nv % kKvSlots, j == 0);
-                        if (j + 1 < n_steps) {
-                            if (x == 0 && !wait_or_abort(&kv_full[nk % kKvSlots], (uint32_t)(nk / kKvSlots) & 1u,
-                                                         abort_flag, wait_limit_ns)) { ok = false; break; }
-                            issue_qk(x, nk % kKvSlots);                // overwrites S_x / P_x after the product above
-                        } else {
-                            umma_commit(leader, &o_done[x]);
-                        }
+                        issue_qk(nk % kKvSlots);
                     }
-                    if (!ok) break;
-                    umma_commit(leader, &kv_empty[nv % kKvSlots]);
-                    if (j + 1 < n_steps) umma_commit(leader, &kv_empty[nk % kKvSlots]);
+                    if (!wait_or_abort(&kv_full[nv % kKvSlots], (uint32_t)(nv / kKvSlots) & 1u, abort_flag, wait_limit_ns) ||
+                        !wait_or_abort(&p_full[x], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
+                    // In the last step tile A's softmax group clears the V rows past the context before it
+                    // hands P_A over; tile B's product reads the same V tile and has to see that too.
+                    if (x == 1 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN &&
+                        !wait_or_abort(&p_full[0], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    issue_pv(nv % kKvSlots, j == 0);
                 }
                 if (!ok && leader) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
@@ -301,18 +325,21 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
             const int r = threadIdx.x & 127;                         // query row = TMEM lane
             const int q_head = x == 0 ? tile.q_head : tile.q_head_b;
             const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-            const uint32_t col_s = Cfg::kColS + x * 128, col_o = Cfg::kColO + x * 128;
+            const uint32_t col_s = Cfg::kColS, col_p = Cfg::kColP + x * 64, col_o = Cfg::kColO + x * 128;
             const int my_pos = min(tile.pos0 + r, tile.ctx_len - 1); // last key this row attends
             float m_used = -INFINITY, l = 0.f;
             bool ok = true;
             for (int j = 0; j < n_steps; ++j) {
-                // S_x(j) complete; the same commit also covers O_x += P_x V of step j-1
+                // S_x(j) complete: copy this row's 128 scores out and give the region back at once
                 if (!wait_or_abort(&s_full[x], (uint32_t)j & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                 tcgen05_fence_after();
                 uint32_t sreg[4][32];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x32(lane_addr + col_s + c * 32, sreg[c]);
                 tmem_ld_wait();
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_out[x]);
                 const int tok0 = j * kTileN;
                 float mx = -INFINITY;
                 if (tok0 + kTileN - 1 > tile.pos0) {
@@ -335,6 +362,11 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 }
                 // Keep the old reference max unless some row of the warp moved by more than the
                 // threshold: P stays bounded by 2^threshold and O needs no rescale most steps.
+                // P_x and O_x belong to the tensor pipe until O_x += P_x V of the step before is done
+                if (j > 0) {
+                    if (!wait_or_abort(&pv_done[x], (uint32_t)(j - 1) & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
+                    tcgen05_fence_after();
+                }
                 const float m_new = fmaxf(m_used, mx);
                 const bool moved = (m_new - m_used) * scale_log2 > kRescaleThreshold;   // true while m_used = -inf
                 const bool rescale = __any_sync(0xffffffffu, moved);
@@ -346,7 +378,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 }
                 const float ms = m_used * scale_log2;
                 const float2 sc2 = make_float2(scale_log2, scale_log2), nms2 = make_float2(-ms, -ms);
-                float2 sum2 = make_float2(0.f, 0.f);
+                float2 sum2 = make_float2(0.f, 0.f), sum2b = make_float2(0.f, 0.f);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t preg[32];                                  // 64 keys as bf16 pairs
@@ -356,8 +388,8 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         float2 xy = __ffma2_rn(make_float2(__uint_as_float(sreg[2 * c + (i >> 4)][(2 * i) & 31]),
                                                            __uint_as_float(sreg[2 * c + (i >> 4)][(2 * i + 1) & 31])),
                                                sc2, nms2);
-                        // one pair in four goes to the FMA pipe instead of the special-function unit
-                        if ((i & 3) == 3) {
+                        // one pair in eight goes to the FMA pipe instead of the special-function unit
+                        if ((i & 7) == 7) {
                             xy = exp2_poly2(xy);
                         } else {
                             xy.x = exp2_approx(xy.x);
@@ -366,14 +398,14 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                         sum2 = __fadd2_rn(sum2, xy);
                         preg[i] = pack_bf16x2(xy.x, xy.y);
                     }
-                    tmem_st_32x32b_x32(lane_addr + col_s + c * 32, preg);
+                    tmem_st_32x32b_x32(lane_addr + col_p + c * 32, preg);
                 }
-                const float sum = sum2.x + sum2.y;
+                const float sum = (sum2.x + sum2b.x) + (sum2.y + sum2b.y);
                 l = l * alpha + sum;
                 tmem_st_wait();
                 if (x == 0 && j == n_steps - 1 && tile.ctx_len < n_steps * kTileN) {
                     // keys past the context hold no token: clear their V rows so 0 * garbage cannot
-                    // poison O (tile A's group does it; tile B's product is issued after tile A's)
+                    // poison O (tile A's group does it; tile B's issuer waits for tile A's hand-over too)
                     const int nv = kv_seq_v(j, n_steps), s = nv % kKvSlots;
                     if (!wait_or_abort(&kv_full[s], (uint32_t)(nv / kKvSlots) & 1u, abort_flag, wait_limit_ns)) { ok = false; break; }
                     uint8_t *v_tile = smem + Cfg::kOffK + s * Cfg::kKvTileBytes;
@@ -389,7 +421,7 @@ prefill_tcgen05_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&p_full[x]);
             }
-            if (ok && wait_or_abort(&o_done[x], 0, abort_flag, wait_limit_ns)) {
+            if (ok && wait_or_abort(&pv_done[x], (uint32_t)(n_steps - 1) & 1u, abort_flag, wait_limit_ns)) {
                 tcgen05_fence_after();
                 const float inv = 1.f / l;
                 const bool valid = r < tile.rows;
