@@ -178,6 +178,8 @@ typedef struct ap_plan_info {
     int64_t launches_append; /* kernels ap_kv_append launches for this plan */
     int64_t launches_attention; /* kernels ap_attention_iteration launches for this plan */
     int64_t side_by_side;    /* 1 if the decode and prefill kernels of this plan run concurrently */
+    int64_t decode_head_block; /* kv heads one decode item covers: 1, or 4 / 2 (the largest that divides the
+                                  pool's kv heads) when decode is confined to part of the GPU */
 } ap_plan_info;
 int ap_plan_get_info(const ap_plan *plan, ap_plan_info *info);
 
@@ -210,9 +212,9 @@ int ap_plan_predict(const ap_plan *plan, double hbm_gbs, double tensor_tflops, a
  * section:
  *   append_dst    [n_new]             page*16 + slot of every new token row
  *   bt_flat       [n_bt]              used block-table entries, sequences with q_len > 0 concatenated
- *   decode_items  [decode_items][8]   q_row, kv_head, bt_offset, page_begin, page_count, kv_len, part_slot, merge_index
+ *   decode_items  [decode_items][8]   q_row, first kv_head of the item's block, bt_offset, page_begin, page_count, kv_len, part_slot, merge_index
  *   cta_begin     [n_cta_begin]       item range of decode CTA c is [cta_begin[c], cta_begin[c+1])
- *   merge_entries [merge_entries][4]  q_row, kv_head, part_begin, part_count
+ *   merge_entries [merge_entries][4]  q_row, first kv_head of the block, part_begin, part_count
  *   prefill_tiles [prefill_tiles][8]  q_row0, rows, q_head, kv_head, bt_offset, pos0, ctx_len, q_head_b (-1: none)
  * blob: host, capacity_ints >= layout.total_ints, or NULL to query the layout only.
  */
@@ -280,9 +282,9 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
  * ap_attention_iteration asks for.
  *
  * This variant does the same work as ap_attention_iteration but keeps the
- * split-K partials in a fixed array of AP_STATIC_WORKSPACE_BYTES (4 MiB) that
+ * split-K partials in a fixed array of AP_STATIC_WORKSPACE_BYTES (8 MiB) that
  * is part of the library image: every GPU context that loads the library
- * holds those 4 MiB until the process exits, used or not.  The call itself
+ * holds those 8 MiB until the process exits, used or not.  The call itself
  * performs no cudaMalloc / cudaFree and calls no allocating routine; q, out
  * and lse are still the caller's.  (Building the plan is a separate, earlier
  * call; ap_plan_create recycles its upload buffers and only allocates when it
@@ -290,8 +292,9 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
  *
  *  - A plan whose ap_plan_workspace_bytes() exceeds AP_STATIC_WORKSPACE_BYTES
  *    is rejected with AP_ERR_WORKSPACE_TOO_SMALL before anything is launched
- *    (4 MiB covers every plan the planner makes for 148 SMs at head_dim 128
- *    and 8 query heads per kv head, including 131072-token contexts).
+ *    (A plan needs at most 2 partials per decode CTA, each head_dim + 1 floats for
+ *    every query head of a block of up to 4 kv heads: 4.9 MB on 148 SMs at
+ *    head_dim 128 with 8 query heads per kv head, whatever the context lengths.)
  *  - The array's device address is looked up once per device when a pool is
  *    created on it (ap_kv_pool_create, which allocates anyway and must not run
  *    inside a stream capture); that is also when the runtime brings the array
@@ -303,7 +306,7 @@ int ap_attention_iteration(ap_kv_pool *pool, const ap_plan *plan, const void *q,
  *    array and produce garbage; order them, or use ap_attention_iteration with
  *    separate workspaces.
  */
-#define AP_STATIC_WORKSPACE_BYTES (4u << 20)
+#define AP_STATIC_WORKSPACE_BYTES (8u << 20)
 size_t ap_static_workspace_bytes(void);
 int ap_attention_iteration_static(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                                   float *lse, void *stream);

@@ -66,7 +66,7 @@ class PlanInfo(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "n_new", "kv_tokens", "decode_rows", "prefill_seqs", "prefill_pairs", "decode_items",
         "decode_ctas", "merge_entries", "prefill_tiles", "launches_append", "launches_attention",
-        "side_by_side")]
+        "side_by_side", "decode_head_block")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -366,7 +366,7 @@ def static_workspace_bytes() -> int:
 def attention_iteration_static(pool: KVPool, plan: Plan, q, out, lse=None, stream=None) -> None:
     """Same result as :func:`attention_iteration`, for callers that cannot
     allocate device memory and therefore have no workspace to pass: the split-K
-    partials go to a fixed 4 MiB array inside the library.  Plans that need
+    partials go to a fixed 8 MiB array inside the library.  Plans that need
     more raise ``ApError`` (``AP_ERR_WORKSPACE_TOO_SMALL``).  Calls share that
     array, so two of them must not overlap on the GPU."""
     _check(load().ap_attention_iteration_static(pool.handle, plan.handle, _ptr(q), _ptr(out), _ptr(lse),

@@ -235,6 +235,7 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
         ap_kv_pool *hp = new (std::nothrow) ap_kv_pool();
         if (!hp) return AP_ERR_CUDA;
         hp->desc = *desc;
+        hp->head_block = decode_head_block(desc->num_kv_heads);
         hp->sm_count = 148;
         hp->free_list.resize((size_t)desc->num_pages);
         for (int32_t i = 0; i < desc->num_pages; ++i) hp->free_list[(size_t)i] = desc->num_pages - 1 - i;
@@ -249,6 +250,7 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
     ap_kv_pool *p = new (std::nothrow) ap_kv_pool();
     if (!p) return AP_ERR_CUDA;
     p->desc = *desc;
+    p->head_block = decode_head_block(desc->num_kv_heads);
     int rc = AP_OK;
     do {
         if (cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, desc->device) != cudaSuccess) {
@@ -283,9 +285,15 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
         }
         rc = prepare_static_workspace(desc->device);
         if (rc != AP_OK) break;
-        rc = encode_pool_tensor_map(&p->k_map, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
+        rc = encode_pool_tensor_map(&p->k_map, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim, 1);
         if (rc != AP_OK) break;
-        rc = encode_pool_tensor_map(&p->v_map, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim);
+        rc = encode_pool_tensor_map(&p->v_map, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim, 1);
+        if (rc != AP_OK) break;
+        rc = encode_pool_tensor_map(&p->k_map_blk, p->desc.k_base, desc->num_pages, desc->num_kv_heads, desc->head_dim,
+                                    p->head_block);
+        if (rc != AP_OK) break;
+        rc = encode_pool_tensor_map(&p->v_map_blk, p->desc.v_base, desc->num_pages, desc->num_kv_heads, desc->head_dim,
+                                    p->head_block);
         if (rc != AP_OK) break;
         p->free_list.resize((size_t)desc->num_pages);
         for (int32_t i = 0; i < desc->num_pages; ++i) p->free_list[(size_t)i] = desc->num_pages - 1 - i;
@@ -456,12 +464,21 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
         }
     }
 
-    // ---- decode: cut the (row, kv head) page streams into per-CTA item lists
+    // ---- decode: cut the (row, kv head block) page streams into per-CTA item lists
     int max_ctas = std::max(1, pool->sm_count * decode_ctas_per_sm(d));
     const int side_ctas = side_by_side_decode_ctas(pool, b, (int)d, (int)Hkv, G, max_ctas);
     if (side_ctas > 0) max_ctas = side_ctas;
-    constexpr int kItemCost = 2;          // fixed per-item cost, in page units
-    constexpr int kStage = kDecodePagesPerStage;
+    // Costs are counted in (page, kv head) tiles.  An item covers HB kv heads, so a page of it is HB
+    // tiles; a ring stage of the kernel holds kStageTiles tiles = PS pages of an item, and streams are
+    // cut on stage boundaries.
+    // Items span a block of kv heads when decode is confined to part of the GPU (next to prefill):
+    // there an SM's stream is bound by its TMA request rate, and requests of HB tiles lift it from
+    // ~58 to ~90 GB/s.  With the whole GPU decode is HBM-bound at ~41 GB/s per SM either way, and
+    // one kv head per item keeps the partials (and their merge in the kernel's tail) small.
+    const int HB = side_ctas > 0 ? pool->head_block : 1, NB = Hkv / HB;
+    constexpr int kStageTiles = kDecodeTilesPerStage;
+    const int PS = kStageTiles / HB;      // pages of an item per stage
+    constexpr int kItemCost = 3;          // fixed per-item cost (its query load, the hand-over of its result)
     std::vector<DecodeItem> items;
     std::vector<int32_t> cta_begin;
     std::vector<MergeEntry> merges;
@@ -469,38 +486,39 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     if (decode_rows > 0) {
         // One pass with an adaptive share: each list gets (cost still to place) / (lists still to
         // fill), so rounding cuts to stage boundaries and the extra items that cuts create spread over
-        // the lists that follow instead of piling up in a last one.  `left` counts pages plus
+        // the lists that follow instead of piling up in a last one.  `left` counts tiles plus
         // kItemCost per item still to emit.
         int64_t left = 0;
         for (int s = 0; s < B; ++s)
             if (b->q_lens[s] == 1)
-                left += (int64_t)Hkv * (((int64_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize + kItemCost);
-        const int64_t min_share = 2 * kStage + kItemCost;
-        items.reserve((size_t)decode_rows * Hkv + 2 * (size_t)max_ctas);
+                left += (int64_t)NB * ((((int64_t)b->ctx_lens[s] + kPageSize - 1) / kPageSize) * HB + kItemCost);
+        const int64_t min_share = 2 * kStageTiles + kItemCost;
+        items.reserve((size_t)decode_rows * NB + 2 * (size_t)max_ctas);
         cta_begin.reserve((size_t)max_ctas + 1);
         cta_begin.push_back(0);
-        // (+ kStage: about what a list loses to rounding; without it the loss drifts to the last lists)
-        int64_t cap = std::max<int64_t>((left + max_ctas - 1) / max_ctas + kStage, min_share);
+        // (+ kStageTiles: about what a list loses to rounding; without it the loss drifts to the last lists)
+        int64_t cap = std::max<int64_t>((left + max_ctas - 1) / max_ctas + kStageTiles, min_share);
         auto next_cta = [&]() {
             if ((int32_t)items.size() > cta_begin.back()) cta_begin.push_back((int32_t)items.size());
             const int lists_left = max_ctas - ((int)cta_begin.size() - 1);
-            cap = lists_left <= 1 ? INT64_MAX / 2 : std::max<int64_t>((left + lists_left - 1) / lists_left + kStage, min_share);
+            cap = lists_left <= 1 ? INT64_MAX / 2
+                                  : std::max<int64_t>((left + lists_left - 1) / lists_left + kStageTiles, min_share);
         };
         for (int s = 0; s < B; ++s) {
             if (b->q_lens[s] != 1) continue;
             const int32_t cl = b->ctx_lens[s];
             const int32_t pages = (cl + kPageSize - 1) / kPageSize;
-            for (int g = 0; g < Hkv; ++g) {
+            for (int hb = 0; hb < NB; ++hb) {
                 int32_t rem = pages, pb = 0;
                 const size_t first = items.size();
                 while (rem > 0) {
-                    int64_t avail = cap - kItemCost;
-                    if (avail < kStage && avail < rem) { next_cta(); continue; }
+                    const int64_t avail = (cap - kItemCost) / HB;          // pages this list can still take
+                    if (avail < PS && avail < rem) { next_cta(); continue; }
                     int32_t take = (int32_t)std::min<int64_t>(rem, avail);
-                    if (take < rem) take = take / kStage * kStage;
+                    if (take < rem) take = take / PS * PS;
                     DecodeItem it{};
                     it.q_row = row0[(size_t)s];
-                    it.kv_head = g;
+                    it.kv_head = hb * HB;
                     it.bt_offset = bt_off[(size_t)s];
                     it.page_begin = pb;
                     it.page_count = take;
@@ -508,14 +526,14 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
                     it.part_slot = -1;
                     it.merge_index = -1;
                     items.push_back(it);
-                    cap -= take + kItemCost;
+                    cap -= (int64_t)take * HB + kItemCost;
                     pb += take;
                     rem -= take;
-                    left -= take + (rem > 0 ? 0 : kItemCost);   // a cut leaves one more item to emit
-                    if (cap < kItemCost + kStage) next_cta();
+                    left -= (int64_t)take * HB + (rem > 0 ? 0 : kItemCost);   // a cut leaves one more item to emit
+                    if (cap < kItemCost + kStageTiles) next_cta();
                 }
                 if (items.size() - first > 1) {
-                    MergeEntry m{row0[(size_t)s], g, n_slots, (int32_t)(items.size() - first)};
+                    MergeEntry m{row0[(size_t)s], hb * HB, n_slots, (int32_t)(items.size() - first)};
                     merges.push_back(m);
                     for (size_t i = first; i < items.size(); ++i) {
                         items[i].part_slot = n_slots++;
@@ -626,6 +644,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     plan->group = G;
     plan->scale = b->softmax_scale > 0.f ? b->softmax_scale : 1.0f / std::sqrt((float)d);
     plan->n_part_slots = n_slots;
+    plan->head_block = HB;
     plan->d_append_dst = plan->buf.dev + o_append;
     plan->d_bt_flat = plan->buf.dev + o_bt;
     plan->d_items = (const DecodeItem *)(plan->buf.dev + o_items);
@@ -633,8 +652,8 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     plan->d_merge = (const MergeEntry *)(plan->buf.dev + o_merge);
     plan->d_tiles = (const PrefillTile *)(plan->buf.dev + o_tiles);
     plan->ws.o_part_off = 0;
-    plan->ws.lse_part_off = align_up((size_t)n_slots * G * d * sizeof(float), 256);
-    plan->ws.bytes = n_slots ? plan->ws.lse_part_off + align_up((size_t)n_slots * G * sizeof(float), 256) : 0;
+    plan->ws.lse_part_off = align_up((size_t)n_slots * HB * G * d * sizeof(float), 256);
+    plan->ws.bytes = n_slots ? plan->ws.lse_part_off + align_up((size_t)n_slots * HB * G * sizeof(float), 256) : 0;
 
     ap_plan_info &info = plan->info;
     info.n_new = n_new;
@@ -667,6 +686,7 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     }
     plan->side_by_side = side_ctas > 0 && !items.empty() && !tiles.empty();
     info.side_by_side = plan->side_by_side ? 1 : 0;
+    info.decode_head_block = HB;
     *out = plan;
     return AP_OK;
 }
@@ -919,8 +939,9 @@ int ap_serving_iteration_host(ap_kv_pool *pool, const ap_batch_desc *batch, cons
     const size_t lse_bytes = align_up(n * Hq * 4, 256);
     // every decode CTA leaves at most two partials, which bounds the workspace before planning
     const size_t max_slots = 2 * (size_t)std::max(1, pool->sm_count * decode_ctas_per_sm((int)d));
-    const size_t ws_bytes = align_up(max_slots * (Hq / Hkv) * d * sizeof(float), 256) +
-                            align_up(max_slots * (Hq / Hkv) * sizeof(float), 256);
+    const size_t part_heads = (size_t)pool->head_block * (Hq / Hkv);      // query heads of one decode item
+    const size_t ws_bytes = align_up(max_slots * part_heads * d * sizeof(float), 256) +
+                            align_up(max_slots * part_heads * sizeof(float), 256);
     const size_t total = 2 * q_bytes + 2 * kv_bytes + lse_bytes + ws_bytes;
     if (total > pool->stage_bytes) {
         if (pool->stage_dev) {

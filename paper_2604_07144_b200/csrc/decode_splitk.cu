@@ -1,20 +1,23 @@
 // Decode attention: split-K flash-decoding over paged KV (HBM-bound).
 //
-// A persistent CTA walks its list of work items; an item is the G query heads
-// of one kv head of one decode row over a contiguous range of the sequence's
-// pages.  One producer warp streams (page, kv head) tiles of K and V -- 4 KB
-// each, contiguous in HBM -- into a multi-stage shared-memory ring with TMA
-// (128-byte swizzle, completion on mbarriers) and runs ahead across item
-// boundaries, so the pipeline never drains while consumers finish an item.
-// Eight consumer warps work as two groups of four that take alternate stages of
-// the ring (two warps per scheduler hide each other's MMA and shuffle latency);
-// within its group's stage a warp owns one page:
+// A persistent CTA walks its list of work items; an item is the query heads of a
+// block of HB consecutive kv heads (HB = 4, 2 or 1) of one decode row over a
+// contiguous range of the sequence's pages.  One producer warp streams K and V
+// into a multi-stage shared-memory ring with TMA (128-byte swizzle, completion on
+// mbarriers), one request per page and plane for the HB (page, kv head) tiles
+// that lie together in HBM (16 KB at HB = 4, d = 128: the TMA unit of an SM
+// sustains ~58 GB/s in 4 KB requests but over 100 GB/s in 16 KB ones), and runs
+// ahead across item boundaries, so the pipeline never drains while consumers
+// finish an item.  Eight consumer warps work as two groups of four that take
+// alternate stages of the ring (two warps per scheduler hide each other's MMA and
+// shuffle latency); a stage holds four tiles per plane (4 / HB pages of HB heads)
+// and within its group's stage a warp owns one (page, kv head) tile:
 //     S^T = K_page Q^T      (mma.sync m16n8k16: M = 16 tokens, N = 8 heads)
 //     online softmax over tokens (fp32, warp shuffles across the token lanes)
 //     O^T += V_page^T P^T   (M = 16 columns of d per tile, N = 8 heads)
 // so every MMA row is a real token and no accumulator register is padding.
-// At the end of an item the four warps drop their (m, l, O) into one of two
-// shared-memory buffers and move on; a combine warp folds them and writes either
+// At the end of an item the eight warps drop their (m, l, O) into a
+// shared-memory buffer and move on; a combine warp folds those of the same kv head and writes either
 // the final bf16 output (item covers the whole context) or an fp32 partial
 // (o normalised, lse), off the consumers' critical path.  A further warp counts the
 // CTA's partials in on a device-wide arrival counter per cut stream; the last
@@ -33,26 +36,37 @@ using namespace ptx;
 
 constexpr int kConsumerWarps = 8;           // two groups of four; a group takes every other stage of the ring
 constexpr int kDecodeThreads = (kConsumerWarps + 3) * 32;   // consumers, producer, LSE-merge warp, combine warp
-constexpr int kPPS = kDecodePagesPerStage;
+constexpr int kTPS = kDecodeTilesPerStage;   // tiles of one plane per stage
 // A stream is only ever cut at a CTA boundary, so a CTA holds at most two items
 // that produce partials (the planner puts them first in the CTA's list).
 constexpr int kMaxPartialItems = 2;
-constexpr int kSmemItems = 64;           // item descriptors of a CTA kept in shared memory
-static_assert(2 * kPPS == kConsumerWarps, "one page of a stage per warp of a consumer group");
+constexpr int kSmemItems = 32;           // item descriptors of a CTA kept in shared memory
+constexpr int kMaxItemHeads = 32;        // query heads of an item: at most 4 kv heads x 8 query heads each
+static_assert(2 * kTPS == kConsumerWarps, "one tile of a stage per warp of a consumer group");
 
 template <int D>
 struct DecodeCfg {
     static constexpr int kTileBytes = kPageSize * D * 2;            // one (page, head) tile of one plane
-    static constexpr int kQBytes = 8 * D * 2;                       // up to 8 query heads
-    static constexpr int kStageBytes = 2 * kPPS * kTileBytes + kQBytes;
-    static constexpr int kStages = D == 128 ? 4 : 8;
+    static constexpr int kStageBytes = 2 * kTPS * kTileBytes;       // K tiles, then V tiles
     static constexpr int kORow = D + 4;                             // padded fp32 row of the merge buffer
     static constexpr int kMergeWarpFloats = 8 * kORow + 16;         // O[8][D+4], m[8], l[8]
-    static constexpr int kMergeBytes = 2 * kConsumerWarps * kMergeWarpFloats * 4;   // two buffers
-    static constexpr int kBarrierBytes = (2 * kStages + kMaxPartialItems + 4) * 8 + 16 + kSmemItems * 32;
-    static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kMergeBytes + kBarrierBytes;
+    static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4;      // one hand-over buffer
+    static constexpr int kQBytes = kMaxItemHeads * D * 2;           // the query heads of one item; two buffers
+    // Two ways to spend the same shared memory (the kernel takes the pair as arguments):
+    //   whole-GPU decode, one kv head per item: many short items, so two hand-over buffers keep the
+    //     consumers from waiting on the combine warp; 4 stages of 32 KB are plenty at ~41 GB/s per SM;
+    //   decode confined to k SMs, a block of kv heads per item: few long items, one buffer will do; the
+    //     ring gets a 5th stage, because an SM's rate is (bytes in flight) / (memory latency) and two
+    //     stages are always held by the consumer groups.
+    static constexpr int kStagesMax = (D == 128 ? 5 : 10);
+    static constexpr int kStagesWide = (D == 128 ? 4 : 8);
+    static constexpr int kBarrierBytes = (2 * kStagesMax + kMaxPartialItems + 8) * 8 + 16 + kSmemItems * 32;
+    static constexpr int kRingAndBuffers = kStagesMax * kStageBytes + kMergeBytes > kStagesWide * kStageBytes + 2 * kMergeBytes
+                                               ? kStagesMax * kStageBytes + kMergeBytes
+                                               : kStagesWide * kStageBytes + 2 * kMergeBytes;
+    static constexpr int kSmemBytes = 1024 + kRingAndBuffers + 2 * kQBytes + kBarrierBytes;
+    static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of an SM");
     static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte swizzle alignment");
-    static_assert(kStages % 2 == 0, "consumer groups own alternate ring slots");
 };
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
@@ -76,18 +90,21 @@ __device__ __forceinline__ uint32_t tile_off(int tok, int chunk) {
 // travel by shuffle, and the o rows are fetched a batch of up to 16 independent 16-byte loads per lane at
 // a time (lane = 4 columns of d).  Streams of more than 32 partials take the same path in chunks,
 // re-reading the lse values from L2 instead of keeping them in registers.
+// A partial holds PH heads (those of the item's kv head block); one call merges G of them, heads
+// h0 .. h0 + G - 1 of the partial, which are query heads first_q_head + h0 ... of the row.
 template <int D, int G>
 __device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o_part, const float *lse_part,
-                                             __nv_bfloat16 *out, float *lse_out, int Hq, int lane) {
+                                             __nv_bfloat16 *out, float *lse_out, int Hq, int lane, int PH, int h0,
+                                             int first_q_head) {
     const int n = me.part_count;
-    const float *lse_base = lse_part + (size_t)me.part_begin * G;
+    const float *lse_base = lse_part + (size_t)me.part_begin * PH + h0;
     // ---- lse of the whole stream, per head
     float v[G], mx[G], sm[G], lse_tot[G];
 #pragma unroll
     for (int h = 0; h < G; ++h) mx[h] = -INFINITY;
     for (int k0 = 0; k0 < n; k0 += 32) {
 #pragma unroll
-        for (int h = 0; h < G; ++h) v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * G + h) : -INFINITY;
+        for (int h = 0; h < G; ++h) v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * PH + h) : -INFINITY;
 #pragma unroll
         for (int h = 0; h < G; ++h) mx[h] = fmaxf(mx[h], v[h]);
     }
@@ -101,7 +118,7 @@ __device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o
         if (n > 32) {
 #pragma unroll
             for (int h = 0; h < G; ++h)
-                v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * G + h) : -INFINITY;
+                v[h] = k0 + lane < n ? __ldcg(lse_base + (size_t)(k0 + lane) * PH + h) : -INFINITY;
         }
 #pragma unroll
         for (int h = 0; h < G; ++h) sm[h] += __expf(v[h] - mx[h]);
@@ -118,13 +135,13 @@ __device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o
 #pragma unroll
     for (int h = 0; h < G; ++h) acc[h] = make_float4(0.f, 0.f, 0.f, 0.f);
     const bool col_ok = lane * 4 < D;
-    const float4 *o_base = reinterpret_cast<const float4 *>(o_part + (size_t)me.part_begin * G * D) + lane;
+    const float4 *o_base = reinterpret_cast<const float4 *>(o_part + ((size_t)me.part_begin * PH + h0) * D) + lane;
     for (int c0 = 0; c0 < n; c0 += 32) {
         float w[G];                                    // this lane's partial (c0 + lane): weight per head
         if (n > 32) {
 #pragma unroll
             for (int h = 0; h < G; ++h)
-                v[h] = c0 + lane < n ? __ldcg(lse_base + (size_t)(c0 + lane) * G + h) : -INFINITY;
+                v[h] = c0 + lane < n ? __ldcg(lse_base + (size_t)(c0 + lane) * PH + h) : -INFINITY;
         }
 #pragma unroll
         for (int h = 0; h < G; ++h) w[h] = __expf(v[h] - lse_tot[h]);
@@ -136,7 +153,7 @@ __device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o
 #pragma unroll
                 for (int h = 0; h < G; ++h)
                     o[kk][h] = (k0 + kk < cn && col_ok)
-                                   ? __ldcg(o_base + ((size_t)(c0 + k0 + kk) * G + h) * (D / 4))
+                                   ? __ldcg(o_base + ((size_t)(c0 + k0 + kk) * PH + h) * (D / 4))
                                    : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int kk = 0; kk < kBatch; ++kk)
@@ -151,10 +168,61 @@ __device__ __forceinline__ void merge_stream(const MergeEntry me, const float *o
 #pragma unroll
     for (int h = 0; h < G; ++h) {
         if (col_ok) {
-            const size_t orow = (size_t)me.q_row * Hq + (size_t)me.kv_head * G + h;
+            const size_t orow = (size_t)me.q_row * Hq + (size_t)(first_q_head + h0 + h);
             *reinterpret_cast<uint2 *>(out + orow * D + lane * 4) =
                 make_uint2(pack_bf16x2(acc[h].x, acc[h].y), pack_bf16x2(acc[h].z, acc[h].w));
             if (lane == 0 && lse_out) lse_out[orow] = lse_tot[h];
+        }
+    }
+}
+
+// Folds, for one item, the consumer warps' (m, l, O) per kv head of the item's block (HB heads; the
+// 8 / HB warps hh, hh + HB, ... worked on head hh) and writes the bf16 output or the fp32 partial.
+template <int D, int HB>
+__device__ __forceinline__ void combine_item(const DecodeItem item, const float *mb, int G, int Hq, float scale_log2,
+                                             __nv_bfloat16 *out, float *lse_out, float *o_part, float *lse_part, int lane) {
+    using Cfg = DecodeCfg<D>;
+    constexpr int kWarpsPerHead = kConsumerWarps / HB;
+    const float kLn2 = 0.6931471805599453f;
+    const bool col_ok = lane * 4 < D;
+    const int PH = HB * G;
+#pragma unroll
+    for (int hh = 0; hh < HB; ++hh) {
+#pragma unroll
+        for (int h = 0; h < 8; ++h) {
+            if (h >= G) break;
+            float mw[kWarpsPerHead], mstar = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < kWarpsPerHead; ++i) {
+                mw[i] = mb[(hh + i * HB) * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + h];
+                mstar = fmaxf(mstar, mw[i]);
+            }
+            float L = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < kWarpsPerHead; ++i) {
+                const float *wb = mb + (hh + i * HB) * Cfg::kMergeWarpFloats;
+                const float wt = exp2_approx((mw[i] - mstar) * scale_log2);
+                L += wt * wb[8 * Cfg::kORow + 8 + h];
+                if (col_ok) {
+                    const float4 o = *reinterpret_cast<const float4 *>(wb + h * Cfg::kORow + lane * 4);
+                    acc.x += wt * o.x; acc.y += wt * o.y; acc.z += wt * o.z; acc.w += wt * o.w;
+                }
+            }
+            const float inv = 1.f / L;
+            const float lse = (mstar * scale_log2 + log2f(L)) * kLn2;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+            if (item.part_slot < 0) {
+                const size_t row = (size_t)item.q_row * Hq + (size_t)(item.kv_head + hh) * G + h;
+                if (col_ok)
+                    *reinterpret_cast<uint2 *>(out + row * D + lane * 4) =
+                        make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
+                if (lane == 0 && lse_out) lse_out[row] = lse;
+            } else {
+                const size_t row = (size_t)item.part_slot * PH + hh * G + h;
+                if (col_ok) *reinterpret_cast<float4 *>(o_part + row * D + lane * 4) = acc;
+                if (lane == 0) lse_part[row] = lse;
+            }
         }
     }
 }
@@ -165,27 +233,32 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                      const __nv_bfloat16 *__restrict__ q, const DecodeItem *__restrict__ items,
                      const int32_t *__restrict__ cta_begin, const int32_t *__restrict__ bt_flat,
                      const MergeEntry *__restrict__ merges, float *o_part, float *lse_part,
-                     __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out, int Hq, int Hkv, int G,
-                     int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns) {
+                     __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out, int Hq, int Hkv, int G, int HB,
+                     int n_stages, int n_bufs, int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns) {
     using Cfg = DecodeCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *stages = smem;
-    float *merge = (float *)(smem + Cfg::kStages * Cfg::kStageBytes);
-    uint64_t *full = (uint64_t *)((uint8_t *)merge + Cfg::kMergeBytes);
-    uint64_t *empty = full + Cfg::kStages;
-    uint64_t *part_done = empty + Cfg::kStages;      // [kMaxPartialItems], each completes once
-    uint64_t *item_done = part_done + kMaxPartialItems;   // [2] consumers -> combine warp, per merge buffer
+    float *merge = (float *)(smem + n_stages * Cfg::kStageBytes);    // [n_bufs] hand-over buffers
+    uint8_t *q_buf = (uint8_t *)merge + n_bufs * Cfg::kMergeBytes;   // [2][kQBytes]
+    uint64_t *full = (uint64_t *)(q_buf + 2 * Cfg::kQBytes);
+    uint64_t *empty = full + Cfg::kStagesMax;
+    uint64_t *part_done = empty + Cfg::kStagesMax;   // [kMaxPartialItems], each completes once
+    uint64_t *item_done = part_done + kMaxPartialItems;   // [2] consumers -> combine warp, per hand-over buffer
     uint64_t *buf_free = item_done + 2;                    // [2] combine warp -> consumers
-    volatile int *abort_flag = (volatile int *)(buf_free + 2);
-    DecodeItem *s_items = (DecodeItem *)(buf_free + 4);
+    uint64_t *q_full = buf_free + 2;                       // [2] an item's query heads have landed
+    uint64_t *q_empty = q_full + 2;                        // [2] all consumer warps have taken their fragments
+    volatile int *abort_flag = (volatile int *)(q_empty + 2);
+    DecodeItem *s_items = (DecodeItem *)(q_empty + 4);
     int *merge_counters = status + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int item_begin = cta_begin[blockIdx.x], item_end = cta_begin[blockIdx.x + 1];
+    const int PS = kTPS / HB;        // pages of an item per stage
+    const int PH = HB * G;           // query heads of an item (and of a partial)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < Cfg::kStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
@@ -193,6 +266,8 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         for (int i = 0; i < 2; ++i) {
             mbar_init(&item_done[i], kConsumerWarps);
             mbar_init(&buf_free[i], 1);
+            mbar_init(&q_full[i], 1);
+            mbar_init(&q_empty[i], kConsumerWarps);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -212,8 +287,14 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
     griddep_launch_dependents();
     if (warp != kConsumerWarps) griddep_wait();
 
-    int stage = 0;
+    // Ring position: stage slot, phase of its barriers, and which consumer group the stage belongs to
+    // (stages go to the two groups in turn, whatever the number of slots).
+    int stage = 0, turn = 0;
     uint32_t phase = 0;
+    auto advance = [&]() {
+        if (++stage == n_stages) { stage = 0; phase ^= 1; }
+        turn ^= 1;
+    };
 
     if (warp == kConsumerWarps) {
         // ------------------------------------------------------ producer --
@@ -224,9 +305,26 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         DecodeItem item = get_item(item_begin);
         int32_t cur = lane < item.page_count ? __ldg(bt_flat + item.bt_offset + item.page_begin + lane) : 0;
         griddep_wait();      // after the first block-table entries are on their way
+        const uint32_t page_bytes = (uint32_t)(2 * HB * Cfg::kTileBytes);   // K and V tiles of one page of the block
         for (int it = item_begin; it < item_end; ++it) {
             const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
             const int npages = item.page_count;
+            {
+                // the item's query heads (PH * D contiguous bf16) go ahead of its first stage, into the
+                // buffer the item before last used
+                const int ti = it - item_begin, qb = ti & 1;
+                if (!wait_or_abort(&q_empty[qb], (((uint32_t)ti >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
+                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    *abort_flag = 1;
+                    return;
+                }
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&q_full[qb], (uint32_t)(PH * D * 2));
+                    bulk_load(q_buf + qb * Cfg::kQBytes, q + ((size_t)item.q_row * Hq + (size_t)item.kv_head * G) * D,
+                              (uint32_t)(PH * D * 2), &q_full[qb]);
+                }
+                __syncwarp();
+            }
             // block-table entries of the next item's first pages are fetched one item ahead
             DecodeItem next_item = item;
             int32_t next_cur = 0;
@@ -238,34 +336,28 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             for (int p0 = 0; p0 < npages; p0 += 32) {
                 const int32_t nxt = p0 + 32 + lane < npages ? __ldg(bt + p0 + 32 + lane) : 0;
                 const int ngroup = min(32, npages - p0);
-                for (int s0 = 0; s0 < ngroup; s0 += kPPS) {
-                    const int n = min(kPPS, ngroup - s0);
+                for (int s0 = 0; s0 < ngroup; s0 += PS) {
+                    const int n = min(PS, ngroup - s0);
                     if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag, wait_limit_ns)) {
                         atomicCAS(status, 0, AP_ERR_TIMEOUT);
                         *abort_flag = 1;
                         return;
                     }
-                    int32_t page = __shfl_sync(0xffffffffu, cur, s0 + (lane & (kPPS - 1)));
-                    const bool first = p0 == 0 && s0 < 2 * kPPS;   // each consumer group reads Q from its first stage
+                    int32_t page = __shfl_sync(0xffffffffu, cur, s0 + (lane & (PS - 1)));
                     uint8_t *st = stages + stage * Cfg::kStageBytes;
-                    if (lane == 0)
-                        mbar_arrive_expect_tx(&full[stage], (uint32_t)(n * 2 * Cfg::kTileBytes +
-                                                                      (first ? G * D * 2 : 0)));
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], (uint32_t)n * page_bytes);
                     __syncwarp();
                     if (lane < n) {
                         if (page < 0 || page >= num_pages) {
                             atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
                             page = 0;
                         }
+                        // one request per plane: the HB tiles of this page that belong to the item's kv heads
                         const int group = (page * Hkv + item.kv_head) * 2;
-                        tma_load_4d(st + lane * Cfg::kTileBytes, &k_map, &full[stage], 0, 0, 0, group);
-                        tma_load_4d(st + (kPPS + lane) * Cfg::kTileBytes, &v_map, &full[stage], 0, 0, 0, group);
-                    } else if (lane == kPPS && first) {
-                        bulk_load(st + 2 * kPPS * Cfg::kTileBytes,
-                                  q + ((size_t)item.q_row * Hq + (size_t)item.kv_head * G) * D,
-                                  (uint32_t)(G * D * 2), &full[stage]);
+                        tma_load_4d(st + lane * HB * Cfg::kTileBytes, &k_map, &full[stage], 0, 0, 0, group);
+                        tma_load_4d(st + (kTPS + lane * HB) * Cfg::kTileBytes, &v_map, &full[stage], 0, 0, 0, group);
                     }
-                    if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+                    advance();
                 }
                 cur = nxt;
             }
@@ -302,70 +394,42 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             }
             last = __shfl_sync(0xffffffffu, last, 0);
             if (!last) continue;
-            switch (G) {
-                case 1: merge_stream<D, 1>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 2: merge_stream<D, 2>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 3: merge_stream<D, 3>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 4: merge_stream<D, 4>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 5: merge_stream<D, 5>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 6: merge_stream<D, 6>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                case 7: merge_stream<D, 7>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
-                default: merge_stream<D, 8>(me, o_part, lse_part, out, lse_out, Hq, lane); break;
+            // the PH heads of the stream, up to eight per pass (what one warp can keep in registers)
+            const int fq = me.kv_head * G;
+            int h0 = 0;
+            for (; h0 + 8 <= PH; h0 += 8) merge_stream<D, 8>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq);
+            switch (PH - h0) {
+                case 1: merge_stream<D, 1>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 2: merge_stream<D, 2>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 3: merge_stream<D, 3>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 4: merge_stream<D, 4>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 5: merge_stream<D, 5>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 6: merge_stream<D, 6>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                case 7: merge_stream<D, 7>(me, o_part, lse_part, out, lse_out, Hq, lane, PH, h0, fq); break;
+                default: break;
             }
         }
         return;
     }
 
     if (warp == kConsumerWarps + 2) {
-        // ---- combine warp: per item, folds the four consumer warps' (m, l, O) into one result,
+        // ---- combine warp: per item and kv head of its block, folds the (m, l, O) of the consumer
+        // warps that worked on that head (warps hh, hh + HB, ...) into one result,
         //   m* = max_w m_w,  L = sum_w 2^((m_w - m*) c) l_w,  o = sum_w 2^((m_w - m*) c) O_w / L,
         // and writes the final bf16 output (item covers the whole context) or the fp32 partial.
-        const float kLn2 = 0.6931471805599453f;
-        const bool col_ok = lane * 4 < D;
         for (int it = item_begin; it < item_end; ++it) {
             const DecodeItem item = get_item(it);
-            const int ti = it - item_begin, buf = ti & 1;
-            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti >> 1) & 1u, abort_flag, wait_limit_ns)) {
+            const int ti = it - item_begin, buf = ti % n_bufs;
+            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti / n_bufs) & 1u, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
-            const float *mb = merge + buf * kConsumerWarps * Cfg::kMergeWarpFloats;
-#pragma unroll
-            for (int h = 0; h < 8; ++h) {
-                if (h >= G) break;
-                float mw[kConsumerWarps], mstar = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    mw[w] = mb[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + h];
-                    mstar = fmaxf(mstar, mw[w]);
-                }
-                float L = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float wt = exp2_approx((mw[w] - mstar) * scale_log2);
-                    L += wt * mb[w * Cfg::kMergeWarpFloats + 8 * Cfg::kORow + 8 + h];
-                    if (col_ok) {
-                        const float4 o = *reinterpret_cast<const float4 *>(mb + w * Cfg::kMergeWarpFloats +
-                                                                            h * Cfg::kORow + lane * 4);
-                        acc.x += wt * o.x; acc.y += wt * o.y; acc.z += wt * o.z; acc.w += wt * o.w;
-                    }
-                }
-                const float inv = 1.f / L;
-                const float lse = (mstar * scale_log2 + log2f(L)) * kLn2;
-                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-                if (item.part_slot < 0) {
-                    const size_t row = (size_t)item.q_row * Hq + (size_t)item.kv_head * G + h;
-                    if (col_ok)
-                        *reinterpret_cast<uint2 *>(out + row * D + lane * 4) =
-                            make_uint2(pack_bf16x2(acc.x, acc.y), pack_bf16x2(acc.z, acc.w));
-                    if (lane == 0 && lse_out) lse_out[row] = lse;
-                } else {
-                    const size_t row = (size_t)item.part_slot * G + h;
-                    if (col_ok) *reinterpret_cast<float4 *>(o_part + row * D + lane * 4) = acc;
-                    if (lane == 0) lse_part[row] = lse;
-                }
+            const float *mb = merge + buf * (Cfg::kMergeBytes / 4);
+            switch (HB) {
+                case 4: combine_item<D, 4>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
+                case 2: combine_item<D, 2>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
+                default: combine_item<D, 1>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
             }
             __syncwarp();
             if (lane == 0) {
@@ -379,7 +443,8 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
 
     // ---------------------------------------------------------- consumers --
     const int g = lane >> 2, t = lane & 3;
-    const int grp = warp / kPPS, slot = warp % kPPS;
+    const int grp = warp / kTPS, slot = warp % kTPS;
+    const int my_head = slot % HB, my_pg = slot / HB;      // this warp's tile in a stage: kv head of the block, page of the stage
 
     for (int it = item_begin; it < item_end; ++it) {
         const DecodeItem item = get_item(it);
@@ -390,10 +455,27 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
         float o[D / 16][4];
 #pragma unroll
         for (int i = 0; i < D / 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        // Q^T as the B operand: b0 = Q[head g][16ks + 2t, +1], b1 = Q[head g][16ks + 8 + 2t, +1], for the G query
+        // heads of this warp's kv head; taken once per item from the buffer the producer filled
         uint32_t qf[D / 16][2];
-        bool have_q = false;
+        {
+            const int ti = it - item_begin, qb = ti & 1;
+            if (!wait_or_abort(&q_full[qb], ((uint32_t)ti >> 1) & 1u, abort_flag, wait_limit_ns)) {
+                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                *abort_flag = 1;
+                return;
+            }
+            const uint32_t *qs = reinterpret_cast<const uint32_t *>(q_buf + qb * Cfg::kQBytes) + ((my_head * G * D) >> 1);
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                qf[ks][0] = g < G ? qs[(g * D + ks * 16 + 2 * t) >> 1] : 0u;
+                qf[ks][1] = g < G ? qs[(g * D + ks * 16 + 8 + 2 * t) >> 1] : 0u;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&q_empty[qb]);
+        }
 
-        for (int p0 = 0; p0 < npages; p0 += kPPS) {
+        for (int p0 = 0; p0 < npages; p0 += PS) {
             // Every warp passes through every stage, also the other group's: it sees the stage
             // arrive and signs it off.  A stage is refilled only after all eight warps are past it,
             // which keeps every waiter within one phase of each barrier (a parity wait is ambiguous
@@ -403,27 +485,17 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                 *abort_flag = 1;
                 return;
             }
-            if ((stage & 1) != grp) {                    // the other group's stage (ring slots alternate)
+            if (turn != grp) {                           // the other group's stage
                 if (lane == 0) mbar_arrive(&empty[stage]);
-                if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+                advance();
                 continue;
             }
             uint8_t *st = stages + stage * Cfg::kStageBytes;
-            if (!have_q) {                               // this group's first stage of the item (it carries Q)
-                have_q = true;
-                // Q^T as the B operand: b0 = Q[head g][16ks + 2t, +1], b1 = Q[head g][16ks + 8 + 2t, +1]
-                const uint32_t *qs = (const uint32_t *)(st + 2 * kPPS * Cfg::kTileBytes);
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    qf[ks][0] = g < G ? qs[(g * D + ks * 16 + 2 * t) >> 1] : 0u;
-                    qf[ks][1] = g < G ? qs[(g * D + ks * 16 + 8 + 2 * t) >> 1] : 0u;
-                }
-            }
-            const int my_page = p0 + slot;
+            const int my_page = p0 + my_pg;
             if (my_page < npages) {
                 const int tv = min(kPageSize, valid - my_page * kPageSize);   // valid tokens in this page (>= 1)
                 const uint32_t k_tile = smem_u32(st + slot * Cfg::kTileBytes);
-                uint8_t *v_ptr = st + (kPPS + slot) * Cfg::kTileBytes;
+                uint8_t *v_ptr = st + (kTPS + slot) * Cfg::kTileBytes;
                 const uint32_t v_tile = smem_u32(v_ptr);
                 if (tv < kPageSize) {
                     // slots past the context hold no token: clear their V rows so 0 * garbage cannot poison O
@@ -484,18 +556,18 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty[stage]);
-            if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+            advance();
         }
 
-        // ---- hand (m, l, O) to the combine warp through one of two shared-memory buffers and go on
-        // with the next item; the buffer is reused two items later, once the combine warp has freed it
-        const int ti = it - item_begin, buf = ti & 1;
-        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
+        // ---- hand (m, l, O) to the combine warp through a shared-memory buffer and go on with the
+        // next item; a buffer is free again once the combine warp has folded the item that used it
+        const int ti = it - item_begin, buf = ti % n_bufs;
+        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
             atomicCAS(status, 0, AP_ERR_TIMEOUT);
             *abort_flag = 1;
             return;
         }
-        float *my_merge = merge + (buf * kConsumerWarps + warp) * Cfg::kMergeWarpFloats;
+        float *my_merge = merge + buf * (Cfg::kMergeBytes / 4) + warp * Cfg::kMergeWarpFloats;
 #pragma unroll
         for (int sh = 4; sh <= 16; sh <<= 1) {
             l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
@@ -534,9 +606,11 @@ cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const v
     const float scale_log2 = plan->scale * 1.4426950408889634f;
     cudaError_t e = launch_overlapped(
         decode_splitk_kernel<D>, (unsigned)plan->info.decode_ctas, (unsigned)kDecodeThreads, (size_t)Cfg::kSmemBytes,
-        stream, pool->k_map, pool->v_map, (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
+        stream, plan->head_block > 1 ? pool->k_map_blk : pool->k_map, plan->head_block > 1 ? pool->v_map_blk : pool->v_map,
+        (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
         plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads,
-        plan->group, pool->desc.num_pages, scale_log2, pool->d_status, pool->wait_limit_ns);
+        plan->group, plan->head_block, plan->head_block > 1 ? Cfg::kStagesMax : Cfg::kStagesWide,
+        plan->head_block > 1 ? 1 : 2, pool->desc.num_pages, scale_log2, pool->d_status, pool->wait_limit_ns);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

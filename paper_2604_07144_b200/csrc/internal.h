@@ -19,11 +19,13 @@ constexpr int kMaxMergeEntries = 4096;   // arrival counters kept per pool (the 
 
 // ---- device work lists (all int32, uploaded as one blob per plan) ---------
 
-// One split-K decode work item: the G query heads of one kv head of one decode
-// row over a contiguous range of that sequence's logical pages.
+// One split-K decode work item: the query heads of one block of kv heads (HB consecutive kv heads,
+// HB = decode_head_block(Hkv), i.e. HB * G query heads) of one decode row over a contiguous range of
+// that sequence's logical pages.  The HB (page, kv head) tiles of a page lie next to one another in a
+// pool plane, so a page costs the decode kernel one TMA request of HB tiles per plane.
 struct DecodeItem {
     int32_t q_row;       // row in q / out
-    int32_t kv_head;
+    int32_t kv_head;     // first kv head of the block
     int32_t bt_offset;   // offset of the sequence's first block-table entry in bt_flat
     int32_t page_begin;  // first logical page of the range
     int32_t page_count;  // pages in the range (>= 1)
@@ -33,10 +35,10 @@ struct DecodeItem {
 };
 static_assert(sizeof(DecodeItem) == 32, "DecodeItem layout");
 
-// One (row, kv head) result assembled from several partials.
+// One (row, kv head block) result assembled from several partials.
 struct MergeEntry {
     int32_t q_row;
-    int32_t kv_head;
+    int32_t kv_head;     // first kv head of the block
     int32_t part_begin;
     int32_t part_count;
 };
@@ -56,8 +58,8 @@ struct PrefillTile {
 };
 static_assert(sizeof(PrefillTile) == 32, "PrefillTile layout");
 
-// Partial buffers inside the caller's workspace: o_part [slots][G][d] fp32
-// followed by lse_part [slots][G] fp32.
+// Partial buffers inside the caller's workspace: o_part [slots][HB * G][d] fp32
+// followed by lse_part [slots][HB * G] fp32.
 struct WorkspaceLayout {
     size_t o_part_off = 0;
     size_t lse_part_off = 0;
@@ -91,7 +93,9 @@ struct ap_kv_pool {
     int sm_count = 0;
     int *d_status = nullptr;          // [0] status word, [1 ..] arrival counters of the merge entries
     uint64_t wait_limit_ns = ap::kDefaultWaitLimitNs;   // bound of every wait inside a kernel
-    CUtensorMap k_map{}, v_map{};
+    CUtensorMap k_map{}, v_map{};          // box = one (page, kv head) tile (prefill)
+    CUtensorMap k_map_blk{}, v_map_blk{};  // box = the head_block tiles of a page that lie together (decode)
+    int head_block = 1;                    // HB: kv heads per decode item
     // allocator
     std::vector<int32_t> free_list;     // pages handed out from the back
     std::vector<uint8_t> allocated;     // per page
@@ -116,6 +120,7 @@ struct ap_plan {
     ap::PlanBuffer buf{};
     int num_q_heads = 0;
     int group = 0;               // G = Hq / Hkv
+    int head_block = 1;          // HB: kv heads per decode item of this plan (1, or the pool's head_block)
     float scale = 0.f;
     ap_plan_info info{};
     ap_plan_layout layout{};
@@ -176,10 +181,16 @@ int prepare_static_workspace(int device);
 
 // Decode kernel launch geometry (used by the planner to size the item lists).
 int decode_ctas_per_sm(int head_dim);
-constexpr int kDecodePagesPerStage = 4;
+constexpr int kDecodeTilesPerStage = 4;    // (page, kv head) tiles of one plane in a ring stage: one per warp of a consumer group
+// kv heads per decode item: the largest of 4, 2, 1 that divides the number of kv heads.  A stage then holds
+// kDecodeTilesPerStage / HB pages of HB heads each.
+inline int decode_head_block(int num_kv_heads) {
+    return num_kv_heads % 4 == 0 ? 4 : num_kv_heads % 2 == 0 ? 2 : 1;
+}
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no libcuda link).
-int encode_pool_tensor_map(CUtensorMap *map, void *base, int num_pages, int num_kv_heads, int head_dim);
+int encode_pool_tensor_map(CUtensorMap *map, void *base, int num_pages, int num_kv_heads, int head_dim,
+                           int tiles_per_box);
 int encode_q_tensor_map(CUtensorMap *map, const void *q, int64_t n_rows, int num_q_heads, int head_dim);
 
 }  // namespace ap

@@ -40,14 +40,18 @@ EncodeTiledFn encode_fn() {
 // A box of (64, 8, d/64, 2) is one (page, kv head) tile.  With the 128-byte
 // swizzle it lands in shared memory as [group][half][8 tokens][64], each
 // [8][64] block being one 1024-byte swizzle atom: the canonical operand layout
-// of tcgen05.mma, and bank-conflict-free for ldmatrix.
-int encode_pool_tensor_map(CUtensorMap *map, void *base, int num_pages, int num_kv_heads, int head_dim) {
+// of tcgen05.mma, and bank-conflict-free for ldmatrix.  A box of
+// (64, 8, d/64, 2 * tiles_per_box) is that many consecutive tiles (the kv heads
+// of one page that follow one another in memory) in one request, laid out tile
+// after tile.
+int encode_pool_tensor_map(CUtensorMap *map, void *base, int num_pages, int num_kv_heads, int head_dim,
+                           int tiles_per_box) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return AP_ERR_CUDA;
     const cuuint64_t halves = (cuuint64_t)head_dim / 64;
     cuuint64_t dims[4] = {64, 8, halves, (cuuint64_t)num_pages * (cuuint64_t)num_kv_heads * 2};
     cuuint64_t strides[3] = {(cuuint64_t)head_dim * 2, 128, (cuuint64_t)head_dim * 2 * 8};
-    cuuint32_t box[4] = {64, 8, (cuuint32_t)halves, 2};
+    cuuint32_t box[4] = {64, 8, (cuuint32_t)halves, 2u * (cuuint32_t)tiles_per_box};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

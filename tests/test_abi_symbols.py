@@ -57,5 +57,5 @@ def test_header_is_plain_c_and_struct_sizes_match_the_binding(tmp_path):
     got = [int(x) for x in subprocess.check_output([str(exe)]).split()]
     want = [ctypes.sizeof(binding.PoolDesc), ctypes.sizeof(binding.BatchDesc), ctypes.sizeof(binding.PlanInfo),
             ctypes.sizeof(binding.PlanPrediction), ctypes.sizeof(binding.PlanLayout), ctypes.sizeof(binding.KernelTimes),
-            len(binding.KERNEL_NAMES), binding.AP_ERR_UNSUPPORTED, 4 << 20]
+            len(binding.KERNEL_NAMES), binding.AP_ERR_UNSUPPORTED, 8 << 20]
     assert got == want

@@ -347,14 +347,14 @@ def test_decode_stream_cut_into_more_than_32_partials():
 
 
 def test_decode_more_items_per_cta_than_the_shared_memory_list_holds():
-    """1500 short decode rows x 8 kv heads = 12 000 items, ~81 per CTA: past the 64 item descriptors a
+    """1500 short decode rows x 8 kv heads = 12 000 items, ~81 per CTA: past the 32 item descriptors a
     CTA keeps in shared memory, so the rest come from global memory.  Every output against the oracle."""
     rng = np.random.default_rng(11)
     b = decode_batch(110, W.SHAPE_8B, rng.integers(1, 49, size=1500))
     run = GpuRun(b)
     try:
         ex = ap.plan_export(run.plan)
-        assert int(np.diff(ex["cta_begin"]).max()) > 64, "no CTA holds more than 64 items"
+        assert int(np.diff(ex["cta_begin"]).max()) > 32, "no CTA holds more than 32 items"
     finally:
         run.close()
     err, lerr = check_batch_full(b)
@@ -544,7 +544,7 @@ def test_config5_trace_parity(budget, chunk):
     from paper_2604_07144_b200.trace_runner import TraceRun
     full_iters, longest_list = _trace_full_check_iterations(budget, chunk)
     if budget == 8192:
-        assert longest_list > 64      # the trace's largest plan overflows a CTA's shared-memory item list
+        assert longest_list > 32      # the trace's largest plan overflows a CTA's shared-memory item list
     run = TraceRun(iterations=200, token_budget=budget, chunk=chunk)
     hq, hkv, d = run.shape
     k_ref = np.full((run.num_pages, hkv, 16, d), W.CANARY, np.uint16)

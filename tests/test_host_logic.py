@@ -95,8 +95,9 @@ def test_plan_validation():
 
 
 def check_plan_coverage(batch: W.Batch, side_by_side=None):
-    """Every (decode row, kv head, page) appears in exactly one item; merge
-    entries and part slots are consistent; every prefill row/head is in one tile."""
+    """Every (decode row, kv head, page) appears in exactly one item (an item covers a block of
+    HB = 4, 2 or 1 consecutive kv heads); merge entries and part slots are consistent; every prefill
+    row/head is in one tile."""
     hq, hkv, d = batch.num_q_heads, batch.num_kv_heads, batch.head_dim
     pool = ap.kv_pool_create(batch.num_pages, hkv, d, device=-1)
     if side_by_side is not None:
@@ -105,6 +106,8 @@ def check_plan_coverage(batch: W.Batch, side_by_side=None):
     ex = ap.plan_export(plan)
     info = ex["info"]
     rows = batch.q_indptr
+    hb = info["decode_head_block"]
+    assert hb == ((4 if hkv % 4 == 0 else 2 if hkv % 2 == 0 else 1) if info["side_by_side"] else 1)
     assert info["n_new"] == batch.n_new and info["kv_tokens"] == batch.kv_tokens
     # append destinations
     exp = []
@@ -119,22 +122,23 @@ def check_plan_coverage(batch: W.Batch, side_by_side=None):
     row_to_seq = {int(rows[s]): s for s in range(batch.batch) if batch.q_lens[s] == 1}
     for q_row, kvh, bt_off, pb, pc, kv_len, slot, _ in items:
         s = row_to_seq[int(q_row)]
-        assert kv_len == batch.ctx_lens[s] and pc >= 1 and 0 <= kvh < hkv
+        assert kv_len == batch.ctx_lens[s] and pc >= 1 and 0 <= kvh < hkv and kvh % hb == 0
         npages = (int(batch.ctx_lens[s]) + 15) // 16
         assert 0 <= pb and pb + pc <= npages
         if pb + pc < npages:
-            assert pc % 4 == 0                      # cuts fall on stage boundaries
+            assert pc % (4 // hb) == 0              # cuts fall on stage boundaries (4 tiles = 4 / HB pages)
         assert list(ex["bt_flat"][bt_off:bt_off + npages]) == list(batch.block_tables[s, :npages])
         for pg in range(pb, pb + pc):
-            assert (s, int(kvh), pg) not in seen
-            seen[(s, int(kvh), pg)] = int(slot)
+            for head in range(int(kvh), int(kvh) + hb):
+                assert (s, head, pg) not in seen
+                seen[(s, head, pg)] = int(slot)
     want = {(s, g, pg) for s in row_to_seq.values() for g in range(hkv)
             for pg in range((int(batch.ctx_lens[s]) + 15) // 16)}
     assert set(seen) == want
     if len(items):
         assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) > 0).all()
         assert len(cta) - 1 == info["decode_ctas"] <= 148
-        cost = [int(items[a:b, 4].sum()) for a, b in zip(cta[:-1], cta[1:])]
+        cost = [int(items[a:b, 4].sum()) * hb for a, b in zip(cta[:-1], cta[1:])]      # in (page, kv head) tiles
         if sum(cost) >= 148 * 64:                   # enough work to balance
             assert max(cost) <= 1.15 * (sum(cost) / len(cost)) + 8
     # merge entries
@@ -201,7 +205,7 @@ def test_side_by_side_planning():
     assert off["side_by_side"] == 0 and off["decode_ctas"] == 148
     forced = check_plan_coverage(b3, side_by_side=40)
     assert forced["side_by_side"] == 1 and forced["decode_ctas"] <= 40
-    assert forced["decode_items"] >= off["decode_rows"] * 8
+    assert forced["decode_items"] >= off["decode_rows"] * 2      # two blocks of four kv heads per row
     for b in (W.config2(with_pool=False), W.config4(with_pool=False)):
         assert check_plan_coverage(b, side_by_side=64)["side_by_side"] == 0
     # a mixed batch too small to gain anything stays sequential under the cost model

@@ -5,7 +5,7 @@ Some integrations run attention from a place where cudaMalloc is off limits:
 all device memory already belongs to a framework's caching allocator, or the
 loop cannot afford cudaMalloc's device-wide synchronisation.  They have no
 workspace to hand to ap_attention_iteration, so the library offers a variant
-that keeps the split-K partials in a fixed 4 MiB array of its own.
+that keeps the split-K partials in a fixed 8 MiB array of its own.
 
 This test drives that variant through the C ABI and requires the same output
 as the ordinary entry point on two calls in a row (the second call sees the
@@ -67,7 +67,7 @@ def _same(got, ref):
 
 
 def test_static_workspace_matches_caller_workspace_twice_in_a_row():
-    assert ap.static_workspace_bytes() == 4 << 20
+    assert ap.static_workspace_bytes() == 8 << 20
     # long contexts: every (row, kv head) stream is cut, so partials and the merge are exercised
     a = GpuRun(_decode_batch(901, [20000, 9001, 333, 64]))
     b = GpuRun(_decode_batch(902, [15000, 12000, 17]))
@@ -122,7 +122,7 @@ def test_static_workspace_with_a_mixed_plan_run_side_by_side():
 def test_static_workspace_small_plan_and_argument_checks():
     # A plan with no cut stream needs no scratch at all and must work too; bad
     # arguments are refused before anything is launched.  (A plan larger than
-    # the 4 MiB array cannot be produced by the planner on 148 SMs, so the
+    # the 8 MiB array cannot be produced by the planner on 148 SMs, so the
     # size rule is checked on the plan's own number.)
     run = GpuRun(_decode_batch(903, [40, 700]))
     try:
