@@ -438,6 +438,8 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
         pools.append(ap.kv_pool_create(batch.num_pages, hkv, d, kp, vp, device=local_rank))
         if side_by_side is not None:
             ap.kv_pool_set_side_by_side(pools[-1], side_by_side)
+        if args.two_streams:
+            ap.kv_pool_set_single_launch(pools[-1], False)
         plans.append(ap.plan_create(pools[-1], batch.q_lens, batch.ctx_lens, batch.block_tables, hq))
     info = ap.plan_get_info(plans[0])
     q, k_new, v_new = dev_bf16(batch.q), dev_bf16(batch.k_new), dev_bf16(batch.v_new)
@@ -559,7 +561,7 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
         kernels = {name: {"launches": n, "us_per_launch": (1e3 * ms / n if n else None)} for name, (ms, n) in kt.items()}
         dec_us = kernels.get("decode_splitk", {}).get("us_per_launch")
         pre_us = kernels.get("prefill", {}).get("us_per_launch")
-        fus_us = kernels.get("fused_mixed", {}).get("us_per_launch")
+        fus_us = kernels.get("mixed_iteration", {}).get("us_per_launch")
         # the profile sums cover this rank's launches only
         achieved = alg["decode_kernel"] / (dec_us * 1e-6) / 1e9 if dec_us else 0.0
         decode_roofline = {
@@ -601,7 +603,8 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
             "config": {"workload": batch.name, "num_q_heads": hq, "num_kv_heads": hkv, "head_dim": d,
                        "page_size": 16, "sequences": batch.batch, "new_tokens": batch.n_new,
                        "kv_tokens_per_step_per_gpu": batch.kv_tokens,
-                       "dispatch": ("fused" if fus_us else "side_by_side" if info["side_by_side"] else "sequential"),
+                       "dispatch": ("one launch: decode CTAs + prefill units" if fus_us else
+                                    "two streams: decode beside prefill" if info["side_by_side"] else "sequential"),
                        "l2": f"rotation among {copies} pool copies ({copies * kv_bytes / 1e9:.2f} GB of KV, each step's "
                              f"{kv_bytes / 1e6:.0f} MB larger than the 126 MB L2)",
                        "timed_region": f"{repeats} x {args.steps} steps back to back ({ms_total:.0f} ms), sized from the warm-up "
@@ -672,6 +675,8 @@ def main():
                           "prefill chunk) and score each by the paper's trace completion time on measured iterations")
     ap_.add_argument("--page-copy", action="store_true",
                      help="time ap_kv_copy_pages on config 2's used pages instead of the serving iteration")
+    ap_.add_argument("--two-streams", action="store_true",
+                     help="mixed iterations: the decode and prefill kernels on two streams instead of one launch")
     ap_.add_argument("--side-by-side", type=int, default=None,
                      help="mixed iterations: 0 = decode then prefill, 1 = planner decides (library default), "
                           "k >= 2 = decode on k CTAs next to prefill")

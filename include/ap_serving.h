@@ -110,16 +110,24 @@ void *ap_kv_pool_v_base(const ap_kv_pool *pool);
 /*
  * Side-by-side execution of mixed iterations (Sec. 5.3: the batch an iteration
  * runs, prefill chunks next to decode tokens, is what the scheduling policy
- * composes).  When a plan holds both decode rows and prefill chunks, the decode
- * kernel can be confined to k persistent CTAs on the caller's stream while the
- * prefill kernel runs at the same time on a stream the pool owns (joined back
- * into the caller's stream before ap_attention_iteration returns control of it).
- * mode 0: never; mode 1 (default): ap_plan_create decides per plan from a cost
- * model and picks k; mode >= 2: always, with k = mode decode CTAs (clamped).
- * Applies to plans created afterwards; results are identical in every mode.
- * ap_plan_info.side_by_side reports what a plan does.  mode < 0 -> INVALID_ARG.
+ * composes).  When a plan holds both decode rows and prefill chunks, decode can
+ * be confined to k persistent CTAs (where it is bound by what an SM can stream,
+ * not by HBM) while the prefill units run on the other SMs at the same time and
+ * take over the decode CTAs' SMs as those retire.  Both parts then go out in ONE
+ * launch on the caller's stream: the decode CTAs are the first k blocks of the
+ * grid, every later block is one prefill unit.
+ * mode 0: never (decode kernel, then prefill kernel); mode 1 (default):
+ * ap_plan_create decides per plan from a cost model and picks k; mode >= 2:
+ * always, with k = mode decode CTAs (clamped).  Applies to plans created
+ * afterwards; results are identical in every mode up to the summation order of
+ * split-K partials.  ap_plan_info.side_by_side reports what a plan does.
+ * mode < 0 -> INVALID_ARG.
  */
 int ap_kv_pool_set_side_by_side(ap_kv_pool *pool, int32_t mode);
+/* on = 0: side-by-side plans use two launches instead, the decode kernel on the caller's stream and the
+ * prefill kernel on a low-priority stream the pool owns, forked and joined with events (kept for
+ * comparison); on != 0 (default): the single launch.  Applies to plans created afterwards. */
+int ap_kv_pool_set_single_launch(ap_kv_pool *pool, int32_t on);
 
 /* Host page allocator (per-request page ownership; pages are relocatable units,
  * Sec. 5.1 Phase 2).  alloc is all-or-nothing: OUT_OF_PAGES leaves the free
@@ -362,9 +370,9 @@ int ap_selftest_wait_timeout(ap_kv_pool *pool, uint64_t limit_ns, int leave_coun
  * launching stream.  ap_profile_collect synchronises `stream`, adds up the
  * elapsed times per kernel since the last enable/collect, and clears the
  * records.  Index: 0 kv_append, 1 decode split-K (which also performs the LSE
- * merge), 2 prefill.
+ * merge), 2 prefill, 3 the single launch that holds both parts of a mixed plan.
  */
-enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_PREFILL = 2, AP_KERNEL_COUNT = 3 };
+enum { AP_KERNEL_APPEND = 0, AP_KERNEL_DECODE = 1, AP_KERNEL_PREFILL = 2, AP_KERNEL_MIXED = 3, AP_KERNEL_COUNT = 4 };
 typedef struct ap_kernel_times {
     double ms[AP_KERNEL_COUNT];
     int64_t launches[AP_KERNEL_COUNT];

@@ -39,7 +39,7 @@ EXPORTED_SYMBOLS = (
     "ap_attention_iteration", "ap_serving_iteration_host", "ap_last_device_status",
     "ap_profile_enable", "ap_profile_collect",
     "ap_static_workspace_bytes", "ap_attention_iteration_static",
-    "ap_kv_pool_set_wait_limit", "ap_selftest_wait_timeout",
+    "ap_kv_pool_set_wait_limit", "ap_selftest_wait_timeout", "ap_kv_pool_set_single_launch",
 )
 
 
@@ -89,10 +89,10 @@ class PlanLayout(ctypes.Structure):
 
 
 class KernelTimes(ctypes.Structure):
-    _fields_ = [("ms", ctypes.c_double * 3), ("launches", ctypes.c_int64 * 3)]
+    _fields_ = [("ms", ctypes.c_double * 4), ("launches", ctypes.c_int64 * 4)]
 
 
-KERNEL_NAMES = ("kv_append", "decode_splitk", "prefill")
+KERNEL_NAMES = ("kv_append", "decode_splitk", "prefill", "mixed_iteration")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -136,6 +136,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
         "ap_profile_collect": (ctypes.c_int, [vp, vp, ctypes.POINTER(KernelTimes)]),
         "ap_static_workspace_bytes": (sz, []),
         "ap_attention_iteration_static": (ctypes.c_int, [vp, vp, vp, vp, vp, vp]),
+        "ap_kv_pool_set_single_launch": (ctypes.c_int, [vp, i32]),
         "ap_kv_pool_set_wait_limit": (ctypes.c_int, [vp, u64]),
         "ap_selftest_wait_timeout": (ctypes.c_int, [vp, u64, ctypes.c_int, vp]),
     }
@@ -246,6 +247,11 @@ def kv_pool_seed_free_list(pool: KVPool, seed: int) -> None:
 def kv_pool_set_side_by_side(pool: KVPool, mode: int) -> None:
     """0: never run decode and prefill concurrently; 1: per-plan decision (default); k >= 2: always, k decode CTAs."""
     _check(load().ap_kv_pool_set_side_by_side(pool.handle, int(mode)), "ap_kv_pool_set_side_by_side")
+
+
+def kv_pool_set_single_launch(pool: KVPool, on: bool) -> None:
+    """Side-by-side plans: one launch for both parts (default) or the decode and prefill kernels on two streams."""
+    _check(load().ap_kv_pool_set_single_launch(pool.handle, int(bool(on))), "ap_kv_pool_set_single_launch")
 
 
 def kv_pool_num_free(pool: KVPool) -> int:

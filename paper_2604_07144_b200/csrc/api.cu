@@ -163,7 +163,12 @@ namespace ap {
 cudaError_t launch_attention_kernels(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
                                      float *o_part, float *lse_part, cudaStream_t st) {
     cudaError_t e = cudaSuccess;
-    if (plan->side_by_side) {
+    if (plan->single_launch) {
+        // One grid: the decode CTAs have the lowest block indices, so they are resident first and the
+        // prefill units fill the remaining SMs and, as decode CTAs retire, those too.
+        TimedScope timed(pool, AP_KERNEL_MIXED, st);
+        e = launch_mixed_iteration(pool, plan, q, out, lse, o_part, lse_part, st);
+    } else if (plan->side_by_side) {
         // Decode goes first, on the caller's stream, so that its few CTAs are resident when the
         // prefill kernel's units (second stream, lower priority) fill the remaining SMs; as decode
         // CTAs retire, prefill units take their SMs too.  The caller's stream continues after both.
@@ -333,6 +338,12 @@ int ap_kv_pool_destroy(ap_kv_pool *pool) {
 int ap_kv_pool_set_side_by_side(ap_kv_pool *pool, int32_t mode) {
     if (!pool || mode < 0) return AP_ERR_INVALID_ARG;
     pool->side_by_side_mode = mode;
+    return AP_OK;
+}
+
+int ap_kv_pool_set_single_launch(ap_kv_pool *pool, int32_t on) {
+    if (!pool) return AP_ERR_INVALID_ARG;
+    pool->single_launch = on != 0;
     return AP_OK;
 }
 
@@ -666,7 +677,6 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     info.merge_entries = (int64_t)merges.size();
     info.prefill_tiles = (int64_t)tiles.size();
     info.launches_append = n_new > 0 ? 1 : 0;
-    info.launches_attention = (items.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
     {
         // algorithmic work of one layer: every attended KV token's K and V once per kv head, q read,
         // out + lse written, used block-table entries once; 4 d flop per (q head, query row, unmasked key)
@@ -685,6 +695,8 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
         plan->work.prefill_sm_us = w_p;
     }
     plan->side_by_side = side_ctas > 0 && !items.empty() && !tiles.empty();
+    plan->single_launch = plan->side_by_side && pool->single_launch;
+    info.launches_attention = plan->single_launch ? 1 : (items.empty() ? 0 : 1) + (tiles.empty() ? 0 : 1);
     info.side_by_side = plan->side_by_side ? 1 : 0;
     info.decode_head_block = HB;
     *out = plan;

@@ -109,6 +109,7 @@ struct ap_kv_pool {
     cudaStream_t side_stream = nullptr;
     cudaEvent_t fork_event = nullptr, join_event = nullptr;
     int side_by_side_mode = 1;        // 0 never, 1 decided per plan, >= 2 that many decode CTAs
+    bool single_launch = true;        // side-by-side plans: one launch for both parts (else two streams)
     // per-kernel event timing (diagnostics)
     bool profiling = false;
     std::vector<ap::TimedLaunch> timed;
@@ -127,7 +128,8 @@ struct ap_plan {
     std::vector<int32_t> blob;   // host copy of the uploaded work lists
     int n_part_slots = 0;
     ap::PlanWork work{};
-    bool side_by_side = false;   // decode on the caller's stream and prefill on the pool's second stream, concurrently
+    bool side_by_side = false;   // decode confined to part of the GPU, prefill on the rest at the same time
+    bool single_launch = false;  // ... and both in one launch (else: two kernels on two streams)
     ap::WorkspaceLayout ws{};
     // device pointers into buf.dev
     const int32_t *d_append_dst = nullptr;
@@ -147,8 +149,12 @@ cudaError_t launch_decode_splitk(const ap_kv_pool *pool, const ap_plan *plan, co
                                  float *lse, float *o_part, float *lse_part, cudaStream_t stream);
 cudaError_t launch_prefill(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out,
                            float *lse, cudaStream_t stream);
+// Both parts of a mixed plan in one launch: the plan's decode CTAs first, then one block per prefill unit.
+cudaError_t launch_mixed_iteration(const ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
+                                   float *o_part, float *lse_part, cudaStream_t stream);
 // Decode and prefill kernels of a plan: one after the other on `stream`, or, for a side-by-side plan,
-// decode on `stream` and prefill on the pool's second stream, joined back into `stream`.
+// both in one launch (or, if the pool asks for it, decode on `stream` and prefill on the pool's second
+// stream, joined back into `stream`).
 cudaError_t launch_attention_kernels(ap_kv_pool *pool, const ap_plan *plan, const void *q, void *out, float *lse,
                                      float *o_part, float *lse_part, cudaStream_t stream);
 // One warp waits on an mbarrier that nothing arrives on, with the given limit (see ap_selftest_wait_timeout).

@@ -25,7 +25,7 @@ def to_bits(t) -> np.ndarray:
 class GpuRun:
     """Pool + plan + device tensors of one batch."""
 
-    def __init__(self, batch: W.Batch, device: int = 0, scale: float = 0.0, side_by_side=None):
+    def __init__(self, batch: W.Batch, device: int = 0, scale: float = 0.0, side_by_side=None, single_launch=None):
         import torch
         self.torch = torch
         self.batch = batch
@@ -43,6 +43,8 @@ class GpuRun:
                                       self.v_pool, device=device)
         if side_by_side is not None:
             ap.kv_pool_set_side_by_side(self.pool, side_by_side)
+        if single_launch is not None:
+            ap.kv_pool_set_single_launch(self.pool, single_launch)
         self.plan = ap.plan_create(self.pool, batch.q_lens, batch.ctx_lens, batch.block_tables,
                                    batch.num_q_heads, softmax_scale=scale)
         self.info = ap.plan_get_info(self.plan)

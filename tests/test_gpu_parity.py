@@ -60,19 +60,22 @@ def test_mixed_ragged_small():
     check_batch_full(W.random_ragged(204, shape=W.SHAPE_8B, batch=5, max_ctx=900, max_q=300))
 
 
-@pytest.mark.parametrize("mode", [0, 3, 20])
-def test_mixed_iteration_side_by_side_modes(mode):
-    """Decode confined to a few CTAs on the caller's stream while prefill runs on the pool's second
-    stream (forced), and the sequential dispatch (mode 0): same results against the oracle, twice in
-    a row on the same pool (its stream and fork / join events are reused)."""
+@pytest.mark.parametrize("mode,single", [(0, True), (3, True), (20, True), (3, False), (20, False)],
+                         ids=["sequential", "k3_one_launch", "k20_one_launch", "k3_two_streams", "k20_two_streams"])
+def test_mixed_iteration_side_by_side_modes(mode, single):
+    """Decode confined to a few CTAs next to the prefill units (forced k) in one launch -- the decode
+    CTAs are the first blocks of the grid, every later block a prefill unit -- or as two kernels on
+    the caller's stream and the pool's second stream, and the sequential dispatch (mode 0): same
+    results against the oracle, twice in a row on the same pool."""
     import oracle
     from harness import compare_outputs, oracle_pools
     batch = W._assemble("mixed_side_by_side", W.SHAPE_8B, W.make_rng(31),
                         np.array([200, 1, 1, 1, 130, 1], np.int32),
                         np.array([700, 333, 1500, 16, 130, 2049], np.int32), 1.3)
-    run = GpuRun(batch, side_by_side=mode)
+    run = GpuRun(batch, side_by_side=mode, single_launch=single)
     try:
         assert run.info["side_by_side"] == (1 if mode else 0)
+        assert run.info["launches_attention"] == (1 if mode and single else 2)
         if mode:
             assert run.info["decode_ctas"] <= mode
         run.append()
@@ -90,8 +93,8 @@ def test_mixed_iteration_side_by_side_modes(mode):
         run.close()
 
 
-@pytest.mark.parametrize("mode", [0, 3])
-def test_iteration_is_capturable_in_a_cuda_graph(mode):
+@pytest.mark.parametrize("mode,single", [(0, True), (3, True), (3, False)], ids=["sequential", "one_launch", "two_streams"])
+def test_iteration_is_capturable_in_a_cuda_graph(mode, single):
     """Append + attention issue no host synchronisation and take every buffer by address, so the
     per-layer sequence of a model (here: the same layer four times) can be captured once into a CUDA
     graph and replayed; with decode beside prefill the fork / join through the pool's second stream
@@ -101,7 +104,7 @@ def test_iteration_is_capturable_in_a_cuda_graph(mode):
     from harness import compare_outputs, oracle_pools
     batch = W._assemble("graph_mixed", W.SHAPE_8B, W.make_rng(41), np.array([150, 1, 1, 1], np.int32),
                         np.array([400, 90, 1300, 17], np.int32), 1.3)
-    run = GpuRun(batch, side_by_side=mode)
+    run = GpuRun(batch, side_by_side=mode, single_launch=single)
     try:
         assert run.info["side_by_side"] == (1 if mode else 0)
         stream = torch.cuda.Stream()
