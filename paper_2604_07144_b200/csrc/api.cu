@@ -85,22 +85,37 @@ cudaEvent_t take_event(ap_kv_pool *pool) {
 }
 
 // Side-by-side execution of a mixed iteration.  Decode is bound by HBM when it has the whole GPU
-// (~41 GB/s per SM at 148 SMs) but one SM's decode pipeline sustains more (~58 GB/s: its ring keeps
-// about 68 KB in flight over a ~1.1 us memory latency), while prefill is bound by the SMs it has.
-// So decode is confined to k SMs, where it is SM-bound, and prefill runs on the others at the same
-// time; the iteration then takes about (W_d + W_p) / #SM, with W the SM-time of each part.  k is
-// the smallest count that lets decode finish within 85 % of that time; beyond ~0.7 #SM decode would
-// be HBM-bound again and nothing is gained, so the plan stays sequential.  The constants were
-// measured on B200 with the 8B attention shape.  Returns 0 for "sequential".
-constexpr double kDecodeSmGBs = 58.0;        // GB/s of KV one SM's decode pipeline sustains
+// (~41 GB/s per SM at 148 SMs) but one SM's decode pipeline sustains more (its ring keeps ~100 KB in
+// flight over a ~1.2 us memory latency; with items that span a block of kv heads the TMA requests are
+// large enough not to be the limit), while prefill is bound by the SMs it has.  So decode is confined
+// to k SMs, where it is SM-bound, and prefill runs on the others at the same time; the iteration then
+// takes about (W_d + W_p) / #SM, with W the SM-time of each part.  k is the smallest count that lets
+// decode finish within 95 % of that time; beyond ~0.7 #SM decode would be HBM-bound again and nothing
+// is gained, so the plan stays sequential.  The constants were measured on B200 (8B and 70B attention
+// shapes, head_dim 128; both kernels running, i.e. at the clocks the power limit leaves: ~1.5 GHz).
+// Returns 0 for "sequential".
+constexpr double kDecodeSmGBs = 68.0;        // GB/s of KV one SM's decode pipeline sustains next to prefill
 constexpr double kDecodeGpuGBs = 6000.0;     // GB/s decode reaches with all SMs
-constexpr double kPrefillStepUs = 2.1;       // one 128-key step of a two-tile unit at d = 128
-constexpr double kPrefillStepSingleUs = 1.5; // the same for a one-tile unit
+constexpr double kPrefillStepUs = 1.9;       // one 128-key step of a two-tile unit at d = 128
+constexpr double kPrefillStepSingleUs = 1.35; // the same for a one-tile unit
 constexpr double kPrefillUnitUs = 5.3;       // prologue + epilogue + relaunch gap of a unit
 constexpr double kPrefillTailUs = 12.0;      // spread of the SMs' finishing times (about half a short unit) + ramp-up
 constexpr double kDecodeFixedUs = 8.0;       // first-data latency and finishing spread of the decode kernel
 constexpr double kAppendGBs = 4000.0;        // scatter of 256-byte rows
 constexpr double kAppendFixedUs = 3.0;
+
+// GB/s of KV one SM's decode pipeline sustains, by the size of its TMA requests (the tiles of one page
+// that an item takes in one request): the TMA unit handles ~14 M requests per second.
+inline double decode_sm_gbs(int request_bytes) {
+    return request_bytes >= 16384 ? kDecodeSmGBs : request_bytes >= 8192 ? 50.0 : request_bytes >= 4096 ? 40.0 : 25.0;
+}
+
+// Time of a mixed iteration with decode on k SMs: decode streams at k times an SM's rate (or what HBM
+// gives), and all SM-time of both parts has to fit on the GPU.
+inline double side_by_side_us(double decode_bytes, double w_p, int k, double sm_rate, int sms) {
+    const double t_dec = decode_bytes / std::min(k * sm_rate, kDecodeGpuGBs * 1e3);
+    return std::max(t_dec, (t_dec * k + w_p) / sms);
+}
 
 int side_by_side_decode_ctas(const ap_kv_pool *pool, const ap_batch_desc *b, int d, int Hkv, int G, int max_ctas) {
     const int mode = pool->side_by_side_mode;
@@ -126,12 +141,15 @@ int side_by_side_decode_ctas(const ap_kv_pool *pool, const ap_batch_desc *b, int
     if (decode_rows == 0 || prefill_seqs == 0) return 0;
     if (mode >= 2) return std::min(mode, max_ctas);
     const int sms = pool->sm_count;
-    const double w_d = decode_bytes / (kDecodeSmGBs * 1e3);              // SM-microseconds
+    const double sm_rate = decode_sm_gbs(pool->head_block * kPageSize * d * 2) * 1e3;      // bytes / us
+    const double w_d = decode_bytes / sm_rate;                                             // SM-microseconds
+    // k that lets decode end with the iteration, at most 0.7 #SM (more would leave prefill too little)
+    int k = (int)std::ceil(w_d / (0.95 * (w_d + w_p) / sms));
+    k = std::max(8, std::min(k, (7 * sms) / 10));
+    if (k >= max_ctas) return 0;
     const double t_serial = decode_bytes / (kDecodeGpuGBs * 1e3) + w_p / sms;
-    const double t_side = (w_d + w_p) / sms;
+    const double t_side = side_by_side_us(decode_bytes, w_p, k, sm_rate, sms);
     if (t_serial - t_side < 10.0 || t_serial - t_side < 0.05 * t_serial) return 0;
-    const int k = (int)std::ceil(w_d / (0.85 * t_side));
-    if (k < 8 || k > (7 * sms) / 10 || k >= max_ctas) return 0;
     return k;
 }
 
@@ -485,8 +503,9 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     // Items span a block of kv heads when decode is confined to part of the GPU (next to prefill):
     // there an SM's stream is bound by its TMA request rate, and requests of HB tiles lift it from
     // ~58 to ~90 GB/s.  With the whole GPU decode is HBM-bound at ~41 GB/s per SM either way, and
-    // one kv head per item keeps the partials (and their merge in the kernel's tail) small.
-    const int HB = side_ctas > 0 ? pool->head_block : 1, NB = Hkv / HB;
+    // one kv head per item keeps the partials (and their merge in the kernel's tail) small -- except at
+    // head_dim 64, where a tile is 2 KB and single-tile requests cannot even feed 148 SMs.
+    const int HB = (side_ctas > 0 || d < 128) ? pool->head_block : 1, NB = Hkv / HB;
     constexpr int kStageTiles = kDecodeTilesPerStage;
     const int PS = kStageTiles / HB;      // pages of an item per stage
     constexpr int kItemCost = 3;          // fixed per-item cost (its query load, the hand-over of its result)
@@ -726,12 +745,15 @@ int ap_plan_predict(const ap_plan *plan, double hbm_gbs, double tensor_tflops, a
     // calibrated model (the one the planner's side-by-side decision uses)
     const int sms = plan->pool->sm_count;
     const double ctas = (double)std::max<int64_t>(plan->info.decode_ctas, 1);
-    const double decode_rate = std::min(ctas * kDecodeSmGBs, kDecodeGpuGBs) * 1e3;        // bytes / us
+    const double decode_rate = std::min(ctas * decode_sm_gbs(plan->head_block * kPageSize * plan->pool->desc.head_dim * 2),
+                                        kDecodeGpuGBs) * 1e3;                             // bytes / us
     e.model_decode_us = w.decode_bytes > 0.0 ? w.decode_bytes / decode_rate + kDecodeFixedUs : 0.0;
     e.model_prefill_us = w.prefill_sm_us > 0.0 ? w.prefill_sm_us / sms + kPrefillTailUs : 0.0;
     const double append_us = w.append_bytes > 0.0 ? w.append_bytes / (kAppendGBs * 1e3) + kAppendFixedUs : 0.0;
     if (plan->side_by_side)
-        e.model_step_us = append_us + (w.decode_bytes / (kDecodeSmGBs * 1e3) + w.prefill_sm_us) / sms + kPrefillTailUs;
+        e.model_step_us = append_us + kPrefillTailUs +
+                          side_by_side_us(w.decode_bytes, w.prefill_sm_us, (int)plan->info.decode_ctas,
+                                          decode_sm_gbs(plan->head_block * kPageSize * plan->pool->desc.head_dim * 2) * 1e3, sms);
     else
         e.model_step_us = append_us + e.model_decode_us + e.model_prefill_us;
     *out = e;

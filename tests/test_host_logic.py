@@ -107,7 +107,8 @@ def check_plan_coverage(batch: W.Batch, side_by_side=None):
     info = ex["info"]
     rows = batch.q_indptr
     hb = info["decode_head_block"]
-    assert hb == ((4 if hkv % 4 == 0 else 2 if hkv % 2 == 0 else 1) if info["side_by_side"] else 1)
+    # a block of kv heads per item when decode is confined to part of the GPU, and always at head_dim 64
+    assert hb == ((4 if hkv % 4 == 0 else 2 if hkv % 2 == 0 else 1) if info["side_by_side"] or d < 128 else 1)
     assert info["n_new"] == batch.n_new and info["kv_tokens"] == batch.kv_tokens
     # append destinations
     exp = []
