@@ -127,7 +127,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "power_w": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -135,7 +135,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
@@ -145,6 +145,10 @@ class ClockSampler:
                     sm.append(float(f[1])); mx.append(float(f[2]))
                 except ValueError:
                     continue
+                try:
+                    pw.append(float(f[3]))
+                except ValueError:
+                    pass
                 for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                     if val.lower().startswith("active"):
                         reasons.add(name)
@@ -152,7 +156,8 @@ class ClockSampler:
         except OSError:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       power_w=(statistics.median(pw) if pw else None))
         return out
 
 
@@ -581,7 +586,11 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
             prefill_roofline = {
                 "bound": "tensor", "kernel": "prefill_tcgen05", "achieved": tf, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": f"of {peaks['source']} (burst)",
-                "frac_of_sustained": tf / peaks["bf16_tflops_sustained"], "frac_of_nominal_2250": tf / 2250.0,
+                "peak_sustained": peaks["bf16_tflops_sustained"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                "which_applies": "the kernel is timed inside a loop of about a second under the power limit (see clocks), "
+                                 "which is the condition of the sustained figure; the burst figure is what a launch "
+                                 "timed alone would be held against",
+                "frac_of_nominal_2250": tf / 2250.0,
                 "traffic": NCU_TRAFFIC.get(("prefill_tcgen05", config, kernel_source_hash("prefill_tcgen05.cu"))),
                 "flops_per_launch": alg["prefill_flops"], "us_per_launch": pre_us,
             }
@@ -631,7 +640,7 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
                                    "model_* = the planner's calibrated cost model; compare model_step_us with ms_per_step"},
             "prefill_tflops": prefill_roofline["achieved"] if prefill_roofline else None,
             "step_gbs": alg["total"] / (ms_per_step * 1e-3) / 1e9,
-            "clocks": ({**{k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples")},
+            "clocks": ({**{k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "power_w")},
                         "ms_x_mhz": (ms_per_step * clocks["sm_mhz"] if clocks["sm_mhz"] else None)} if clocks else None),
         }
     for pl in plans:

@@ -38,9 +38,6 @@ using namespace ptx;
 constexpr int kConsumerWarps = 8;           // two groups of four; a group takes every other stage of the ring
 constexpr int kDecodeThreads = (kConsumerWarps + 3) * 32;   // consumers, producer, LSE-merge warp, combine warp
 constexpr int kTPS = kDecodeTilesPerStage;   // tiles of one plane per stage
-// A stream is only ever cut at a CTA boundary, so a CTA holds at most two items
-// that produce partials (the planner puts them first in the CTA's list).
-constexpr int kMaxPartialItems = 2;
 constexpr int kSmemItems = 32;           // item descriptors of a CTA kept in shared memory
 constexpr int kMaxItemHeads = 32;        // query heads of an item: at most 4 kv heads x 8 query heads each
 static_assert(2 * kTPS == kConsumerWarps, "one tile of a stage per warp of a consumer group");
@@ -51,7 +48,7 @@ struct DecodeCfg {
     static constexpr int kStageBytes = 2 * kTPS * kTileBytes;       // K tiles, then V tiles
     static constexpr int kORow = D + 4;                             // padded fp32 row of the merge buffer
     static constexpr int kMergeWarpFloats = 8 * kORow + 16;         // O[8][D+4], m[8], l[8]
-    static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4;      // one hand-over buffer
+    static constexpr int kMergeBytes = kConsumerWarps * kMergeWarpFloats * 4 + 32; // one hand-over buffer: the warps' data, then the item
     static constexpr int kQBytes = kMaxItemHeads * D * 2;           // the query heads of one item; two buffers
     // Two ways to spend the same shared memory (the kernel takes the pair as arguments):
     //   whole-GPU decode, one kv head per item: many short items, so two hand-over buffers keep the
@@ -61,7 +58,7 @@ struct DecodeCfg {
     //     stages are always held by the consumer groups.
     static constexpr int kStagesMax = (D == 128 ? 5 : 10);
     static constexpr int kStagesWide = (D == 128 ? 4 : 8);
-    static constexpr int kBarrierBytes = (2 * kStagesMax + kMaxPartialItems + 8) * 8 + 16 + kSmemItems * 32;
+    static constexpr int kBarrierBytes = (2 * kStagesMax + 8 + 2) * 8 + 16 + kSmemItems * 32;
     static constexpr int kRingAndBuffers = kStagesMax * kStageBytes + kMergeBytes > kStagesWide * kStageBytes + 2 * kMergeBytes
                                                ? kStagesMax * kStageBytes + kMergeBytes
                                                : kStagesWide * kStageBytes + 2 * kMergeBytes;
@@ -245,17 +242,19 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
     uint8_t *q_buf = (uint8_t *)merge + n_bufs * Cfg::kMergeBytes;   // [2][kQBytes]
     uint64_t *full = (uint64_t *)(q_buf + 2 * Cfg::kQBytes);
     uint64_t *empty = full + Cfg::kStagesMax;
-    uint64_t *part_done = empty + Cfg::kStagesMax;   // [kMaxPartialItems], each completes once
-    uint64_t *item_done = part_done + kMaxPartialItems;   // [2] consumers -> combine warp, per hand-over buffer
+    uint64_t *item_done = empty + Cfg::kStagesMax;         // [2] consumers -> combine warp, per hand-over buffer
     uint64_t *buf_free = item_done + 2;                    // [2] combine warp -> consumers
     uint64_t *q_full = buf_free + 2;                       // [2] an item's query heads have landed
     uint64_t *q_empty = q_full + 2;                        // [2] all consumer warps have taken their fragments
-    volatile int *abort_flag = (volatile int *)(q_empty + 2);
-    DecodeItem *s_items = (DecodeItem *)(q_empty + 4);
+    uint64_t *merge_req = q_empty + 2;                     // combine warp -> merge warp: a stream is complete
+    uint64_t *merge_ack = merge_req + 1;                   // merge warp -> combine warp: request taken care of
+    volatile int *abort_flag = (volatile int *)(merge_ack + 1);
+    volatile int *merge_idx = abort_flag + 1;              // the request: index of the merge entry, or -1: no more
+    DecodeItem *s_items = (DecodeItem *)(merge_ack + 3);   // [kSmemItems] the head of the CTA's list
     int *merge_counters = status + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int item_begin = cta_begin[cta], item_end = cta_begin[cta + 1];
+    const int item_begin = cta_begin[cta], n_items = cta_begin[cta + 1] - item_begin;
     const int PS = kTPS / HB;        // pages of an item per stage
     const int PH = HB * G;           // query heads of an item (and of a partial)
 
@@ -264,25 +263,31 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
-        for (int i = 0; i < kMaxPartialItems; ++i) mbar_init(&part_done[i], 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&item_done[i], kConsumerWarps);
             mbar_init(&buf_free[i], 1);
             mbar_init(&q_full[i], 1);
             mbar_init(&q_empty[i], kConsumerWarps);
         }
+        mbar_init(merge_req, 1);
+        mbar_init(merge_ack, 1);
         *abort_flag = 0;
         fence_barrier_init();
     }
     // The CTA's item descriptors go to shared memory once, so that neither the producer nor the
     // consumers pay a global-memory round trip at every item boundary.
     {
-        const int n_ints = min(item_end - item_begin, kSmemItems) * (int)(sizeof(DecodeItem) / 4);
+        const int n_ints = min(n_items, kSmemItems) * (int)(sizeof(DecodeItem) / 4);
         const int32_t *src = reinterpret_cast<const int32_t *>(items + item_begin);
         for (int i = threadIdx.x; i < n_ints; i += kDecodeThreads) reinterpret_cast<int32_t *>(s_items)[i] = __ldg(src + i);
     }
     named_barrier_sync(1, kDecodeThreads);      // the threads of this role only (the block may hold more)
-    auto get_item = [&](int it) -> DecodeItem { return it - item_begin < kSmemItems ? s_items[it - item_begin] : items[it]; };
+    // Item number n of this CTA's list; page_count 0 past its end.
+    auto get_item = [&](int n) {
+        DecodeItem item{};
+        if (n < n_items) item = n < kSmemItems ? s_items[n] : items[item_begin + n];
+        return item;
+    };
     // Everything up to here reads only the plan (uploaded before the step's kernels), so it may
     // overlap the tail of the kernel before this one; the pool, q, the partial buffers and the
     // counters may not be touched before that kernel is done.
@@ -290,7 +295,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
     if (warp != kConsumerWarps) griddep_wait();
 
     // Ring position: stage slot, phase of its barriers, and which consumer group the stage belongs to
-    // (stages go to the two groups in turn, whatever the number of slots).
+    // (the stages of an item go to the two groups in turn, whatever the number of slots).
     int stage = 0, turn = 0;
     uint32_t phase = 0;
     auto advance = [&]() {
@@ -304,18 +309,21 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
             prefetch_tensormap(&k_map);
             prefetch_tensormap(&v_map);
         }
-        DecodeItem item = get_item(item_begin);
+        DecodeItem item = get_item(0);
         int32_t cur = lane < item.page_count ? __ldg(bt_flat + item.bt_offset + item.page_begin + lane) : 0;
         griddep_wait();      // after the first block-table entries are on their way
         const uint32_t page_bytes = (uint32_t)(2 * HB * Cfg::kTileBytes);   // K and V tiles of one page of the block
-        for (int it = item_begin; it < item_end; ++it) {
+        for (int n = 0; item.page_count > 0; ++n) {
             const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
             const int npages = item.page_count;
+            // the first block-table entries of the next item are fetched one item ahead
+            const DecodeItem next = get_item(n + 1);
+            const int32_t next_cur = lane < next.page_count ? __ldg(bt_flat + next.bt_offset + next.page_begin + lane) : 0;
             {
                 // the item's query heads (PH * D contiguous bf16) go ahead of its first stage, into the
                 // buffer the item before last used
-                const int ti = it - item_begin, qb = ti & 1;
-                if (!wait_or_abort(&q_empty[qb], (((uint32_t)ti >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
+                const int qb = n & 1;
+                if (!wait_or_abort(&q_empty[qb], (((uint32_t)n >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
                     atomicCAS(status, 0, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                     return;
@@ -327,19 +335,11 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 }
                 __syncwarp();
             }
-            // block-table entries of the next item's first pages are fetched one item ahead
-            DecodeItem next_item = item;
-            int32_t next_cur = 0;
-            if (it + 1 < item_end) {
-                next_item = get_item(it + 1);
-                next_cur = lane < next_item.page_count
-                               ? __ldg(bt_flat + next_item.bt_offset + next_item.page_begin + lane) : 0;
-            }
             for (int p0 = 0; p0 < npages; p0 += 32) {
                 const int32_t nxt = p0 + 32 + lane < npages ? __ldg(bt + p0 + 32 + lane) : 0;
                 const int ngroup = min(32, npages - p0);
                 for (int s0 = 0; s0 < ngroup; s0 += PS) {
-                    const int n = min(PS, ngroup - s0);
+                    const int np = min(PS, ngroup - s0);
                     if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag, wait_limit_ns)) {
                         atomicCAS(status, 0, AP_ERR_TIMEOUT);
                         *abort_flag = 1;
@@ -347,9 +347,9 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                     }
                     int32_t page = __shfl_sync(0xffffffffu, cur, s0 + (lane & (PS - 1)));
                     uint8_t *st = stages + stage * Cfg::kStageBytes;
-                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], (uint32_t)n * page_bytes);
+                    if (lane == 0) mbar_arrive_expect_tx(&full[stage], (uint32_t)np * page_bytes);
                     __syncwarp();
-                    if (lane < n) {
+                    if (lane < np) {
                         if (page < 0 || page >= num_pages) {
                             atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
                             page = 0;
@@ -363,39 +363,29 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 }
                 cur = nxt;
             }
-            item = next_item;
+            item = next;
             cur = next_cur;
         }
         return;
     }
 
     if (warp == kConsumerWarps + 1) {
-        // ---- LSE merge warp, off the critical path.  For each of this CTA's partial items, once the
-        // consumers have written it: count it in on the stream's device-wide arrival counter; the
-        // item that completes the count merges all partials of the stream,
+        // ---- LSE merge warp, off everybody's path: when the combine warp has counted in the last
+        // partial of a stream it asks this warp to merge the stream's partials,
         //   lse = m* + ln sum_k exp(lse_k - m*),  o = sum_k exp(lse_k - lse) o_k,  m* = max_k lse_k,
-        // and writes the bf16 result.  mbarrier arrive/wait carry the consumers' stores to this
-        // warp (release/acquire at CTA scope); the acq_rel atomic publishes them device-wide and
-        // acquires the other items' partials.
-        for (int pi = 0; pi < kMaxPartialItems && item_begin + pi < item_end; ++pi) {
-            const DecodeItem item = get_item(item_begin + pi);
-            if (item.part_slot < 0) break;
-            const MergeEntry me = merges[item.merge_index];
-            if (!wait_or_abort(&part_done[pi], 0, abort_flag, wait_limit_ns)) {
+        // and to write the bf16 result.  (The counting atomic is acq_rel at device scope: it publishes
+        // this CTA's partial and acquires the others'; the request barrier carries that on to this warp.)
+        for (uint32_t r = 0;; ++r) {
+            if (!wait_or_abort(merge_req, r & 1u, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
-            int last = 0;
-            if (lane == 0) {
-                int old;
-                asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
-                             : "=r"(old) : "l"(merge_counters + item.merge_index) : "memory");
-                last = old == me.part_count - 1;
-                if (last) merge_counters[item.merge_index] = 0;      // ready for the next launch
-            }
-            last = __shfl_sync(0xffffffffu, last, 0);
-            if (!last) continue;
+            const int idx = *merge_idx;
+            if (idx < 0) return;
+            const MergeEntry me = merges[idx];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(merge_ack);         // the request word may be reused
             // the PH heads of the stream, up to eight per pass (what one warp can keep in registers)
             const int fq = me.kv_head * G;
             int h0 = 0;
@@ -411,34 +401,63 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 default: break;
             }
         }
-        return;
     }
 
     if (warp == kConsumerWarps + 2) {
         // ---- combine warp: per item and kv head of its block, folds the (m, l, O) of the consumer
         // warps that worked on that head (warps hh, hh + HB, ...) into one result,
         //   m* = max_w m_w,  L = sum_w 2^((m_w - m*) c) l_w,  o = sum_w 2^((m_w - m*) c) O_w / L,
-        // and writes the final bf16 output (item covers the whole context) or the fp32 partial.
-        for (int it = item_begin; it < item_end; ++it) {
-            const DecodeItem item = get_item(it);
-            const int ti = it - item_begin, buf = ti % n_bufs;
-            if (!wait_or_abort(&item_done[buf], (uint32_t)(ti / n_bufs) & 1u, abort_flag, wait_limit_ns)) {
+        // and writes the final bf16 output (item covers the whole context) or the fp32 partial.  A
+        // partial is then counted in on its stream's device-wide arrival counter; the one that
+        // completes the count has the merge warp merge the stream.  The item's description comes with
+        // the consumers' data (this warp may be an item or two behind them).
+        uint32_t requests = 0;
+        auto post = [&](int idx) {                // to the merge warp; waits for the request before to be taken
+            if (requests > 0 && !wait_or_abort(merge_ack, (requests - 1) & 1u, abort_flag, wait_limit_ns)) return false;
+            if (lane == 0) {
+                *merge_idx = idx;
+                mbar_arrive(merge_req);
+            }
+            ++requests;
+            return true;
+        };
+        for (int n = 0;; ++n) {
+            const int buf = n % n_bufs;
+            if (!wait_or_abort(&item_done[buf], (uint32_t)(n / n_bufs) & 1u, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
             const float *mb = merge + buf * (Cfg::kMergeBytes / 4);
+            const DecodeItem item = *reinterpret_cast<const DecodeItem *>(mb + kConsumerWarps * Cfg::kMergeWarpFloats);
+            if (item.page_count == 0) break;                       // the consumers are through
             switch (HB) {
                 case 4: combine_item<D, 4>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
                 case 2: combine_item<D, 2>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
                 default: combine_item<D, 1>(item, mb, G, Hq, scale_log2, out, lse_out, o_part, lse_part, lane); break;
             }
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(&buf_free[buf]);
-                // the partial is complete: hand it to the merge warp
-                if (item.part_slot >= 0 && ti < kMaxPartialItems) mbar_arrive(&part_done[ti]);
+            if (lane == 0) mbar_arrive(&buf_free[buf]);
+            if (item.part_slot >= 0) {
+                int last = 0;
+                if (lane == 0) {
+                    int old;
+                    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;"
+                                 : "=r"(old) : "l"(merge_counters + item.merge_index) : "memory");
+                    last = old == __ldg(&merges[item.merge_index].part_count) - 1;
+                    if (last) merge_counters[item.merge_index] = 0;      // ready for the next launch
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last && !post(item.merge_index)) {
+                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    *abort_flag = 1;
+                    return;
+                }
             }
+        }
+        if (!post(-1)) {
+            atomicCAS(status, 0, AP_ERR_TIMEOUT);
+            *abort_flag = 1;
         }
         return;
     }
@@ -448,10 +467,25 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
     const int grp = warp / kTPS, slot = warp % kTPS;
     const int my_head = slot % HB, my_pg = slot / HB;      // this warp's tile in a stage: kv head of the block, page of the stage
 
-    for (int it = item_begin; it < item_end; ++it) {
-        const DecodeItem item = get_item(it);
+    for (int n = 0;; ++n) {
+        const DecodeItem item = get_item(n);
+        const int buf = n % n_bufs;
+        float *hand_over = merge + buf * (Cfg::kMergeBytes / 4);
+        if (item.page_count == 0) {
+            // no more items: tell the combine warp through the hand-over buffer
+            if (!wait_or_abort(&buf_free[buf], ((uint32_t)(n / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
+                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                *abort_flag = 1;
+                return;
+            }
+            if (warp == 0 && lane == 0) *reinterpret_cast<DecodeItem *>(hand_over + kConsumerWarps * Cfg::kMergeWarpFloats) = item;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&item_done[buf]);
+            return;
+        }
         const int npages = item.page_count;
         const int valid = min(item.kv_len, (item.page_begin + npages) * kPageSize) - item.page_begin * kPageSize;
+        turn = 0;    // an item's first stage goes to group 0 whatever came before
 
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
         float o[D / 16][4];
@@ -461,8 +495,8 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         // heads of this warp's kv head; taken once per item from the buffer the producer filled
         uint32_t qf[D / 16][2];
         {
-            const int ti = it - item_begin, qb = ti & 1;
-            if (!wait_or_abort(&q_full[qb], ((uint32_t)ti >> 1) & 1u, abort_flag, wait_limit_ns)) {
+            const int qb = n & 1;
+            if (!wait_or_abort(&q_full[qb], ((uint32_t)n >> 1) & 1u, abort_flag, wait_limit_ns)) {
                 atomicCAS(status, 0, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
@@ -561,15 +595,15 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
             advance();
         }
 
-        // ---- hand (m, l, O) to the combine warp through a shared-memory buffer and go on with the
-        // next item; a buffer is free again once the combine warp has folded the item that used it
-        const int ti = it - item_begin, buf = ti % n_bufs;
-        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(ti / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
+        // ---- hand (m, l, O) and the item's description to the combine warp through a shared-memory
+        // buffer and go on with the next item; a buffer is free again once the combine warp has folded
+        // the item that used it
+        if (!wait_or_abort(&buf_free[buf], ((uint32_t)(n / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
             atomicCAS(status, 0, AP_ERR_TIMEOUT);
             *abort_flag = 1;
             return;
         }
-        float *my_merge = merge + buf * (Cfg::kMergeBytes / 4) + warp * Cfg::kMergeWarpFloats;
+        float *my_merge = hand_over + warp * Cfg::kMergeWarpFloats;
 #pragma unroll
         for (int sh = 4; sh <= 16; sh <<= 1) {
             l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
@@ -588,11 +622,11 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
             my_merge[8 * Cfg::kORow + 8 + 2 * t] = l0;
             my_merge[8 * Cfg::kORow + 8 + 2 * t + 1] = l1;
         }
+        if (warp == 0 && lane == 0) *reinterpret_cast<DecodeItem *>(hand_over + kConsumerWarps * Cfg::kMergeWarpFloats) = item;
         __syncwarp();
         if (lane == 0) mbar_arrive(&item_done[buf]);
     }
 }
-
 
 }  // namespace decode
 }  // namespace ap
