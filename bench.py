@@ -47,13 +47,19 @@ UNIT = "KV-tokens/s"
 # workload (ncu captures summarised under profiles/), keyed by (kernel, config, hash of
 # the kernel's source file the counters were taken from); a changed kernel reports null.
 NCU_TRAFFIC = {
+    # profiles/decode_splitk_config2.md: 536.9 MB read + 5.4 MB written per launch (algorithmic 535.0 MB)
+    ("decode_splitk", 2, "dace136ca989df10"): 542.3e6,
+    # profiles/prefill_tcgen05_config3.md: 148.8 MB read + 18.5 MB written per launch (K/V re-reads are served by the L2)
+    ("prefill_tcgen05", 3, "4c642ed83baf9501"): 167.2e6,
 }
 
 
-def kernel_source_hash(source_file: str) -> str:
+def kernel_source_hash(*source_files: str) -> str:
+    """Hash of the files a kernel's device code lives in (its .cu, the .cuh with the body, the PTX wrappers)."""
     h = hashlib.sha256()
-    with open(os.path.join(ROOT, "paper_2604_07144_b200", "csrc", source_file), "rb") as fh:
-        h.update(fh.read())
+    for f in source_files + ("ptx.cuh",):
+        with open(os.path.join(ROOT, "paper_2604_07144_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
     return h.hexdigest()[:16]
 
 
@@ -572,7 +578,7 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
         decode_roofline = {
             "bound": "hbm", "kernel": "decode_splitk", "achieved": achieved, "peak": peaks["hbm_gbs"],
             "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-            "traffic": NCU_TRAFFIC.get(("decode_splitk", config, kernel_source_hash("decode_splitk.cu"))),
+            "traffic": NCU_TRAFFIC.get(("decode_splitk", config, kernel_source_hash("decode_splitk.cu", "decode_splitk.cuh"))),
             "bytes_per_launch": alg["decode_kernel"], "us_per_launch": dec_us,
             "frac_of_nominal_8TBs": achieved / 8000.0,
         }
@@ -580,6 +586,10 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
         if concurrent:
             decode_roofline["note"] = ("in this plan decode shares the GPU with prefill, so its own time is not a "
                                        "whole-GPU bandwidth figure; see step_roofline")
+        if not dec_us:
+            decode_roofline.update(achieved=None, frac=None, frac_of_nominal_8TBs=None,
+                                   note="no decode kernel of its own in this plan (one launch holds both parts, or the "
+                                        "batch has no decode rows); see step_roofline")
         prefill_roofline = None
         if pre_us:
             tf = alg["prefill_flops"] / (pre_us * 1e-6) / 1e12
@@ -591,7 +601,8 @@ def measure_config(config: int, args, rank: int, world: int, local_rank: int, si
                                  "which is the condition of the sustained figure; the burst figure is what a launch "
                                  "timed alone would be held against",
                 "frac_of_nominal_2250": tf / 2250.0,
-                "traffic": NCU_TRAFFIC.get(("prefill_tcgen05", config, kernel_source_hash("prefill_tcgen05.cu"))),
+                "traffic": NCU_TRAFFIC.get(("prefill_tcgen05", config,
+                                            kernel_source_hash("prefill_tcgen05.cu", "prefill_tcgen05.cuh"))),
                 "flops_per_launch": alg["prefill_flops"], "us_per_launch": pre_us,
             }
             if concurrent:

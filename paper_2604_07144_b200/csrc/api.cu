@@ -580,13 +580,8 @@ int ap_plan_create(ap_plan **out, ap_kv_pool *pool, const ap_batch_desc *b, void
     for (int c = 0; c < n_ctas; ++c)
         std::stable_partition(items.begin() + cta_begin[(size_t)c], items.begin() + cta_begin[(size_t)c + 1],
                               [](const DecodeItem &it) { return it.part_slot >= 0; });
-    // streams are cut at CTA boundaries only, so a CTA has at most two partial items
-    // (the decode kernel relies on it)
-    for (int c = 0; c < n_ctas; ++c) {
-        int partial = 0;
-        for (int32_t i = cta_begin[(size_t)c]; i < cta_begin[(size_t)c + 1]; ++i) partial += items[(size_t)i].part_slot >= 0;
-        if (partial > 2) return AP_ERR_UNSUPPORTED;
-    }
+    // (streams are cut at CTA boundaries only, so a CTA has at most two partial items and the
+    // workspace at most two slots per CTA)
     if ((int)merges.size() > kMaxMergeEntries) return AP_ERR_UNSUPPORTED;
 
     // ---- prefill tiles, longest first

@@ -221,9 +221,9 @@ def test_page_copy_full_size_config2():
 
 @pytest.mark.parametrize("config", [2, 3, 4])
 def test_plan_predict_tracks_the_measured_step(config):
-    """The planner's calibrated model (ap_plan_predict.model_step_us) stays within a factor of the
+    """The planner's calibrated model (ap_plan_predict.model_step_us) stays within -25 % / +35 % of the
     measured device time of append + attention on the full-size workloads, and the paper's roofline
-    time is a lower bound of the measured attention time."""
+    time is a lower bound of the measured attention time (up to the slack explained below)."""
     import torch
     batch = {2: W.config2, 3: W.config3, 4: W.config4}[config]()
     run = GpuRun(batch)
@@ -241,8 +241,12 @@ def test_plan_predict_tracks_the_measured_step(config):
         torch.cuda.synchronize()
         assert run.status() == 0
         us = 1e3 * e0.elapsed_time(e1) / n
-        assert 0.6 * us <= pred["model_step_us"] <= 1.6 * us, (us, pred)
-        # the pool stays in L2 only for small workloads; these are all larger than L2
+        # measured on B200: model / measured = 1.12 (config 2), 0.92 (config 3, one launch), 1.08 (config 4)
+        assert 0.75 * us <= pred["model_step_us"] <= 1.35 * us, (us, pred)
+        # The paper's roofline time is a lower bound in principle, but its B_g here is the bandwidth of a
+        # plain device-to-device copy (6468 GB/s) and the decode kernel, which only reads, streams at up to
+        # 6.97 TB/s on config 4: 1.08x that "peak".  Hence 1.2 and not 1.0.  (These workloads are all much
+        # larger than the L2, so no cache effect is involved.)
         assert max(pred["roofline_decode_us"], pred["roofline_prefill_us"]) <= 1.2 * us
     finally:
         run.close()
