@@ -291,11 +291,14 @@ int ap_kv_pool_create(ap_kv_pool **out, const ap_pool_desc *desc) {
                 break;
             }
         }
-        if (cudaMalloc((void **)&p->d_status, sizeof(int) * (1 + kMaxMergeEntries)) != cudaSuccess ||
-            cudaMemset(p->d_status, 0, sizeof(int) * (1 + kMaxMergeEntries)) != cudaSuccess) {
+        if (cudaMalloc((void **)&p->d_counters, sizeof(int) * kMaxMergeEntries) != cudaSuccess ||
+            cudaMemset(p->d_counters, 0, sizeof(int) * kMaxMergeEntries) != cudaSuccess ||
+            cudaHostAlloc((void **)&p->h_status, sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
+            cudaHostGetDevicePointer((void **)&p->status_dev, p->h_status, 0) != cudaSuccess) {
             rc = AP_ERR_CUDA;
             break;
         }
+        *p->h_status = 0;
         {
             int least = 0, greatest = 0;
             if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess ||
@@ -343,7 +346,8 @@ int ap_kv_pool_destroy(ap_kv_pool *pool) {
     if (pool->fork_event) (void)cudaEventDestroy(pool->fork_event);
     if (pool->join_event) (void)cudaEventDestroy(pool->join_event);
     if (pool->stage_dev) (void)cudaFree(pool->stage_dev);
-    if (pool->d_status) (void)cudaFree(pool->d_status);
+    if (pool->d_counters) (void)cudaFree(pool->d_counters);
+    if (pool->h_status) (void)cudaFreeHost(pool->h_status);
     if (pool->owns_planes) {
         if (pool->desc.k_base) (void)cudaFree(pool->desc.k_base);
         if (pool->desc.v_base) (void)cudaFree(pool->desc.v_base);
@@ -873,15 +877,16 @@ int ap_last_device_status(ap_kv_pool *pool, void *stream) {
     DeviceGuard guard(pool->desc.device);
     if (!guard.ok) return AP_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    int status = 0;
-    if (cudaMemcpyAsync(&status, pool->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
+    // the kernels write the word straight into host memory: after the synchronisation it can be read here
+    if (cudaStreamSynchronize(st) != cudaSuccess) {
         (void)cudaGetLastError();
         return AP_ERR_CUDA;
     }
+    const int status = *reinterpret_cast<volatile int *>(pool->h_status);
     if (status != 0) {
+        *reinterpret_cast<volatile int *>(pool->h_status) = 0;
         // a kernel that gave up may have left merge arrival counters behind: clear them too
-        if (cudaMemsetAsync(pool->d_status, 0, sizeof(int) * (1 + kMaxMergeEntries), st) != cudaSuccess ||
+        if (cudaMemsetAsync(pool->d_counters, 0, sizeof(int) * kMaxMergeEntries, st) != cudaSuccess ||
             cudaStreamSynchronize(st) != cudaSuccess) {
             (void)cudaGetLastError();
             return AP_ERR_CUDA;

@@ -15,9 +15,10 @@ decode_splitk_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_con
                      const int32_t *__restrict__ cta_begin, const int32_t *__restrict__ bt_flat,
                      const MergeEntry *__restrict__ merges, float *o_part, float *lse_part,
                      __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out, int Hq, int Hkv, int G, int HB,
-                     int n_stages, int n_bufs, int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns) {
+                     int n_stages, int n_bufs, int num_pages, float scale_log2, int *status, int *merge_counters,
+                     uint64_t wait_limit_ns) {
     decode_cta<D>(k_map, v_map, q, items, cta_begin, bt_flat, merges, o_part, lse_part, out, lse_out, Hq, Hkv, G, HB, n_stages,
-                  n_bufs, num_pages, scale_log2, status, wait_limit_ns, (int)blockIdx.x);
+                  n_bufs, num_pages, scale_log2, status, merge_counters, wait_limit_ns, (int)blockIdx.x);
 }
 
 template <int D>
@@ -39,7 +40,7 @@ cudaError_t launch_decode_t(const ap_kv_pool *pool, const ap_plan *plan, const v
         (const __nv_bfloat16 *)q, plan->d_items, plan->d_cta_begin, plan->d_bt_flat,
         plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads,
         plan->group, plan->head_block, plan->head_block > 1 ? Cfg::kStagesMax : Cfg::kStagesWide,
-        plan->head_block > 1 ? 1 : 2, pool->desc.num_pages, scale_log2, pool->d_status, pool->wait_limit_ns);
+        plan->head_block > 1 ? 1 : 2, pool->desc.num_pages, scale_log2, pool->status_dev, pool->d_counters, pool->wait_limit_ns);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -233,7 +233,8 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                                            const int32_t *__restrict__ bt_flat, const MergeEntry *__restrict__ merges,
                                            float *o_part, float *lse_part, __nv_bfloat16 *__restrict__ out,
                                            float *__restrict__ lse_out, int Hq, int Hkv, int G, int HB, int n_stages, int n_bufs,
-                                           int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns, int cta) {
+                                           int num_pages, float scale_log2, int *status, int *merge_counters,
+                                           uint64_t wait_limit_ns, int cta) {
     using Cfg = DecodeCfg<D>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -251,7 +252,6 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
     volatile int *abort_flag = (volatile int *)(merge_ack + 1);
     volatile int *merge_idx = abort_flag + 1;              // the request: index of the merge entry, or -1: no more
     DecodeItem *s_items = (DecodeItem *)(merge_ack + 3);   // [kSmemItems] the head of the CTA's list
-    int *merge_counters = status + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int item_begin = cta_begin[cta], n_items = cta_begin[cta + 1] - item_begin;
@@ -324,7 +324,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 // buffer the item before last used
                 const int qb = n & 1;
                 if (!wait_or_abort(&q_empty[qb], (((uint32_t)n >> 1) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
-                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    record_status(status, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                     return;
                 }
@@ -341,7 +341,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 for (int s0 = 0; s0 < ngroup; s0 += PS) {
                     const int np = min(PS, ngroup - s0);
                     if (!wait_or_abort(&empty[stage], phase ^ 1, abort_flag, wait_limit_ns)) {
-                        atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                        record_status(status, AP_ERR_TIMEOUT);
                         *abort_flag = 1;
                         return;
                     }
@@ -351,7 +351,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                     __syncwarp();
                     if (lane < np) {
                         if (page < 0 || page >= num_pages) {
-                            atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                            record_status(status, AP_ERR_BAD_BLOCK_TABLE);
                             page = 0;
                         }
                         // one request per plane: the HB tiles of this page that belong to the item's kv heads
@@ -377,7 +377,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         // this CTA's partial and acquires the others'; the request barrier carries that on to this warp.)
         for (uint32_t r = 0;; ++r) {
             if (!wait_or_abort(merge_req, r & 1u, abort_flag, wait_limit_ns)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
@@ -424,7 +424,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         for (int n = 0;; ++n) {
             const int buf = n % n_bufs;
             if (!wait_or_abort(&item_done[buf], (uint32_t)(n / n_bufs) & 1u, abort_flag, wait_limit_ns)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
@@ -449,14 +449,14 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                 }
                 last = __shfl_sync(0xffffffffu, last, 0);
                 if (last && !post(item.merge_index)) {
-                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    record_status(status, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                     return;
                 }
             }
         }
         if (!post(-1)) {
-            atomicCAS(status, 0, AP_ERR_TIMEOUT);
+            record_status(status, AP_ERR_TIMEOUT);
             *abort_flag = 1;
         }
         return;
@@ -474,7 +474,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         if (item.page_count == 0) {
             // no more items: tell the combine warp through the hand-over buffer
             if (!wait_or_abort(&buf_free[buf], ((uint32_t)(n / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
@@ -497,7 +497,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         {
             const int qb = n & 1;
             if (!wait_or_abort(&q_full[qb], ((uint32_t)n >> 1) & 1u, abort_flag, wait_limit_ns)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
@@ -517,7 +517,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
             // which keeps every waiter within one phase of each barrier (a parity wait is ambiguous
             // beyond that).
             if (!wait_or_abort(&full[stage], phase, abort_flag, wait_limit_ns)) {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
                 return;
             }
@@ -599,7 +599,7 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         // buffer and go on with the next item; a buffer is free again once the combine warp has folded
         // the item that used it
         if (!wait_or_abort(&buf_free[buf], ((uint32_t)(n / n_bufs) & 1u) ^ 1u, abort_flag, wait_limit_ns)) {
-            atomicCAS(status, 0, AP_ERR_TIMEOUT);
+            record_status(status, AP_ERR_TIMEOUT);
             *abort_flag = 1;
             return;
         }

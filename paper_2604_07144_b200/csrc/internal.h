@@ -91,7 +91,9 @@ struct ap_kv_pool {
     ap_pool_desc desc{};
     bool owns_planes = false;
     int sm_count = 0;
-    int *d_status = nullptr;          // [0] status word, [1 ..] arrival counters of the merge entries
+    int *h_status = nullptr;          // the status word: pinned host memory mapped into the device's address space
+    int *status_dev = nullptr;        // ... and the address the kernels write it at
+    int *d_counters = nullptr;        // device: arrival counters of the merge entries
     uint64_t wait_limit_ns = ap::kDefaultWaitLimitNs;   // bound of every wait inside a kernel
     CUtensorMap k_map{}, v_map{};          // box = one (page, kv head) tile (prefill)
     CUtensorMap k_map_blk{}, v_map_blk{};  // box = the head_block tiles of a page that lie together (decode)

@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(uint4 *__restrict__ k_po
     ptx::griddep_wait();                              // the pool may still be read by the kernel before
     const int32_t page = dst >> 4, slot = dst & 15;
     if (page < 0 || page >= num_pages) {
-        atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+        ptx::record_status(status, AP_ERR_BAD_BLOCK_TABLE);
         return;
     }
     const int64_t o = (((int64_t)page * num_kv_heads + g) * kPageSize + slot) * chunks_per_row + c;
@@ -47,7 +47,7 @@ cudaError_t launch_kv_append(const ap_kv_pool *pool, const ap_plan *plan, const 
     cudaError_t e = launch_overlapped(kv_append_kernel, (unsigned)blocks, (unsigned)threads, 0, stream,
                                       (uint4 *)pool->desc.k_base, (uint4 *)pool->desc.v_base, (const uint4 *)k_new,
                                       (const uint4 *)v_new, plan->d_append_dst, n_vec, pool->desc.num_kv_heads, chunks,
-                                      pool->desc.num_pages, pool->d_status);
+                                      pool->desc.num_pages, pool->status_dev);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

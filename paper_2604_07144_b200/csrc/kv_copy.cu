@@ -24,7 +24,7 @@ kv_copy_pages_kernel(uint4 *__restrict__ k_dst, uint4 *__restrict__ v_dst, const
     ptx::griddep_wait();                          // the pools may still be in use by the kernel before
     const int32_t dst = __ldg(pairs + 2 * blockIdx.y), src = __ldg(pairs + 2 * blockIdx.y + 1);
     if (dst < 0 || dst >= num_pages_dst || src < 0 || src >= num_pages_src) {
-        if (threadIdx.x == 0) atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+        if (threadIdx.x == 0) ptx::record_status(status, AP_ERR_BAD_BLOCK_TABLE);
         return;
     }
     const int64_t so = (int64_t)src * page_vecs, dof = (int64_t)dst * page_vecs;
@@ -70,7 +70,7 @@ cudaError_t launch_kv_copy_pages(const ap_kv_pool *dst_pool, const ap_kv_pool *s
         e = cudaLaunchKernelEx(&cfg, kv_copy_pages_kernel, (uint4 *)dst_pool->desc.k_base,
                                (uint4 *)dst_pool->desc.v_base, (const uint4 *)src_pool->desc.k_base,
                                (const uint4 *)src_pool->desc.v_base, d_pairs + 2 * (size_t)done, page_vecs,
-                               (int)dst_pool->desc.num_pages, (int)src_pool->desc.num_pages, dst_pool->d_status);
+                               (int)dst_pool->desc.num_pages, (int)src_pool->desc.num_pages, dst_pool->status_dev);
     }
     return e != cudaSuccess ? e : cudaGetLastError();
 }

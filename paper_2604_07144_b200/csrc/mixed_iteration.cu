@@ -26,13 +26,14 @@ mixed_iteration_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_c
                        const int32_t *__restrict__ bt_flat, const MergeEntry *__restrict__ merges, float *o_part,
                        float *lse_part, __nv_bfloat16 *__restrict__ out, float *__restrict__ lse_out,
                        const PrefillTile *__restrict__ tiles, int Hq, int Hkv, int G, int HB, int n_stages, int n_bufs,
-                       int num_pages, float scale_log2, int *status, uint64_t wait_limit_ns, int n_decode_ctas) {
+                       int num_pages, float scale_log2, int *status, int *merge_counters, uint64_t wait_limit_ns,
+                       int n_decode_ctas) {
     static_assert(decode::kDecodeThreads <= prefill::kPrefillThreads, "the block is sized for the larger role");
     if ((int)blockIdx.x < n_decode_ctas) {
         if (threadIdx.x < decode::kDecodeThreads)
             decode::decode_cta<D>(HB > 1 ? k_map_blk : k_map, HB > 1 ? v_map_blk : v_map, q, items, cta_begin, bt_flat, merges,
                                   o_part, lse_part, out, lse_out, Hq, Hkv, G, HB, n_stages, n_bufs, num_pages, scale_log2,
-                                  status, wait_limit_ns, (int)blockIdx.x);
+                                  status, merge_counters, wait_limit_ns, (int)blockIdx.x);
     } else {
         prefill::prefill_unit<D>(q_map, k_map, v_map, tiles, bt_flat, out, lse_out, Hq, Hkv, num_pages, scale_log2, status,
                                  wait_limit_ns, (int)blockIdx.x - n_decode_ctas);
@@ -61,7 +62,7 @@ cudaError_t launch_mixed_t(const ap_kv_pool *pool, const ap_plan *plan, const vo
         plan->d_cta_begin, plan->d_bt_flat, plan->d_merge, o_part, lse_part, (__nv_bfloat16 *)out, lse, plan->d_tiles,
         plan->num_q_heads, pool->desc.num_kv_heads, plan->group, plan->head_block,
         plan->head_block > 1 ? DCfg::kStagesMax : DCfg::kStagesWide, plan->head_block > 1 ? 1 : 2, pool->desc.num_pages,
-        scale_log2, pool->d_status, pool->wait_limit_ns, (int)plan->info.decode_ctas);
+        scale_log2, pool->status_dev, pool->d_counters, pool->wait_limit_ns, (int)plan->info.decode_ctas);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -38,7 +38,7 @@ cudaError_t launch_prefill_t(const ap_kv_pool *pool, const ap_plan *plan, const 
         prefill_tcgen05_kernel<D>, (unsigned)plan->info.prefill_tiles, (unsigned)kPrefillThreads,
         (size_t)Cfg::kSmemBytes, stream, q_map, pool->k_map, pool->v_map, plan->d_tiles, plan->d_bt_flat,
         (__nv_bfloat16 *)out, lse, plan->num_q_heads, pool->desc.num_kv_heads, pool->desc.num_pages, scale_log2,
-        pool->d_status, pool->wait_limit_ns);
+        pool->status_dev, pool->wait_limit_ns);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -212,7 +212,7 @@ __device__ __forceinline__ void prefill_unit(const CUtensorMap &q_map, const CUt
                 const int np = min(kPagesPerTile, total_pages - j * kPagesPerTile);
                 int32_t page = lane < np ? __ldg(bt + j * kPagesPerTile + lane) : 0;
                 if (!wait_or_abort(&kv_empty[s], ph ^ 1u, abort_flag, wait_limit_ns)) {
-                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    record_status(status, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                     break;
                 }
@@ -220,7 +220,7 @@ __device__ __forceinline__ void prefill_unit(const CUtensorMap &q_map, const CUt
                 __syncwarp();
                 if (lane < np) {
                     if (page < 0 || page >= num_pages) {
-                        atomicCAS(status, 0, AP_ERR_BAD_BLOCK_TABLE);
+                        record_status(status, AP_ERR_BAD_BLOCK_TABLE);
                         page = 0;
                     }
                     const int group = (page * Hkv + tile.kv_head) * 2;
@@ -311,7 +311,7 @@ __device__ __forceinline__ void prefill_unit(const CUtensorMap &q_map, const CUt
                     issue_pv(nv % kKvSlots, j == 0);
                 }
                 if (!ok && leader) {
-                    atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                    record_status(status, AP_ERR_TIMEOUT);
                     *abort_flag = 1;
                 }
             }
@@ -447,7 +447,7 @@ __device__ __forceinline__ void prefill_unit(const CUtensorMap &q_map, const CUt
                     lse_out[(size_t)(tile.q_row0 + r) * Hq + q_head] =
                         (m_used * scale_log2 + log2f(l)) * 0.6931471805599453f;
             } else {
-                atomicCAS(status, 0, AP_ERR_TIMEOUT);
+                record_status(status, AP_ERR_TIMEOUT);
                 *abort_flag = 1;
             }
         }

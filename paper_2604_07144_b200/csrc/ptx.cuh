@@ -16,6 +16,14 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
 
+// The pool's status word lives in pinned host memory that the device can write (so the host reads it
+// after a stream synchronisation without a copy of its own).  Only error paths write it: a plain store,
+// any error code is as good as another when several paths fail at once.
+__device__ __forceinline__ void record_status(int *status, int code) {
+    *reinterpret_cast<volatile int *>(status) = code;
+    __threadfence_system();
+}
+
 // ---------------------------------------------------------------- mbarrier --
 
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {

@@ -13,7 +13,7 @@ namespace ap {
 
 namespace {
 
-__global__ void __launch_bounds__(32) selftest_wait_kernel(int *status, uint64_t limit_ns, int leave_counter) {
+__global__ void __launch_bounds__(32) selftest_wait_kernel(int *status, int *merge_counters, uint64_t limit_ns, int leave_counter) {
     __shared__ uint64_t bar;
     __shared__ int abort_flag;
     if (threadIdx.x == 0) {
@@ -24,10 +24,10 @@ __global__ void __launch_bounds__(32) selftest_wait_kernel(int *status, uint64_t
     __syncwarp();
     // like a decode CTA whose stream's partial was counted in before the CTA gave up: the arrival
     // counter of merge entry 0 is left at 1, which ap_last_device_status has to clear
-    if (leave_counter && threadIdx.x == 0) atomicAdd(status + 1, 1);
+    if (leave_counter && threadIdx.x == 0) atomicAdd(merge_counters, 1);
     if (!ptx::wait_or_abort(&bar, 0, &abort_flag, limit_ns)) {
         if (threadIdx.x == 0) {
-            atomicCAS(status, 0, AP_ERR_TIMEOUT);
+            ptx::record_status(status, AP_ERR_TIMEOUT);
             abort_flag = 1;
         }
     }
@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(32) selftest_wait_kernel(int *status, uint64_t
 }  // namespace
 
 cudaError_t launch_selftest_wait(const ap_kv_pool *pool, uint64_t limit_ns, int leave_counter, cudaStream_t stream) {
-    selftest_wait_kernel<<<1, 32, 0, stream>>>(pool->d_status, limit_ns, leave_counter);
+    selftest_wait_kernel<<<1, 32, 0, stream>>>(pool->status_dev, pool->d_counters, limit_ns, leave_counter);
     return cudaGetLastError();
 }
 
