@@ -22,7 +22,7 @@ def to_bits(t) -> np.ndarray:
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
-class GpuRun:
+class DeviceRun:
     """Pool + plan + device tensors of one batch."""
 
     def __init__(self, batch: W.Batch, device: int = 0, scale: float = 0.0, side_by_side=None, single_launch=None):
@@ -127,7 +127,7 @@ def compare_outputs(out_bits: np.ndarray, lse: np.ndarray, ref_out: np.ndarray, 
 def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None, peaked: bool = False):
     """Append + attention on the GPU against the oracle, every element.  `peaked`: the inputs make the
     softmax nearly one-hot, so the per-element bound of peaked_tolerance replaces the flat one."""
-    run = GpuRun(batch, scale=scale, side_by_side=side_by_side)
+    run = DeviceRun(batch, scale=scale, side_by_side=side_by_side)
     try:
         run.append()
         run.attend()
@@ -152,7 +152,7 @@ def check_batch_full(batch: W.Batch, scale: float = 0.0, side_by_side=None, peak
 def check_batch_sampled(batch: W.Batch, n_samples: int, seed: int = 0):
     """Full-size check: the append is compared bit-exactly on the whole pool,
     attention on randomly sampled (sequence, token, head) outputs."""
-    run = GpuRun(batch)
+    run = DeviceRun(batch)
     try:
         run.append()
         run.attend()

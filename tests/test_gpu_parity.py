@@ -9,7 +9,7 @@ import paper_2604_07144_b200 as ap
 from paper_2604_07144_b200 import binding as B
 from paper_2604_07144_b200 import workloads as W
 
-from harness import GpuRun, check_batch_full, check_batch_sampled, to_bits
+from harness import DeviceRun, check_batch_full, check_batch_sampled, to_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -44,7 +44,7 @@ def test_decode_head_ratios(shape):
 def test_decode_split_and_merge_long_context():
     # few long sequences: every (row, kv head) stream is cut across many CTAs
     b = decode_batch(104, W.SHAPE_8B, [20000, 9001, 333])
-    run = GpuRun(b)
+    run = DeviceRun(b)
     assert run.info["merge_entries"] > 0 and run.info["decode_ctas"] > 100
     run.close()
     check_batch_full(b)
@@ -72,7 +72,7 @@ def test_mixed_iteration_side_by_side_modes(mode, single):
     batch = W._assemble("mixed_side_by_side", W.SHAPE_8B, W.make_rng(31),
                         np.array([200, 1, 1, 1, 130, 1], np.int32),
                         np.array([700, 333, 1500, 16, 130, 2049], np.int32), 1.3)
-    run = GpuRun(batch, side_by_side=mode, single_launch=single)
+    run = DeviceRun(batch, side_by_side=mode, single_launch=single)
     try:
         assert run.info["side_by_side"] == (1 if mode else 0)
         assert run.info["launches_attention"] == (1 if mode and single else 2)
@@ -104,7 +104,7 @@ def test_iteration_is_capturable_in_a_cuda_graph(mode, single):
     from harness import compare_outputs, oracle_pools
     batch = W._assemble("graph_mixed", W.SHAPE_8B, W.make_rng(41), np.array([150, 1, 1, 1], np.int32),
                         np.array([400, 90, 1300, 17], np.int32), 1.3)
-    run = GpuRun(batch, side_by_side=mode, single_launch=single)
+    run = DeviceRun(batch, side_by_side=mode, single_launch=single)
     try:
         assert run.info["side_by_side"] == (1 if mode else 0)
         stream = torch.cuda.Stream()
@@ -150,7 +150,7 @@ def test_page_copy_migration_and_copy_on_write(shape):
     from harness import compare_outputs, to_dev
     batch = W._assemble("migrate", shape, W.make_rng(51), np.array([1, 70, 1, 1, 3], np.int32),
                         np.array([300, 200, 17, 1025, 64], np.int32), 1.3)
-    run = GpuRun(batch)
+    run = DeviceRun(batch)
     try:
         run.append()
         used = _used_pages(batch)
@@ -226,7 +226,7 @@ def test_plan_predict_tracks_the_measured_step(config):
     time is a lower bound of the measured attention time (up to the slack explained below)."""
     import torch
     batch = {2: W.config2, 3: W.config3, 4: W.config4}[config]()
-    run = GpuRun(batch)
+    run = DeviceRun(batch)
     try:
         pred = ap.plan_predict(run.plan)
         for _ in range(3):
@@ -309,7 +309,7 @@ def test_fork_a_sequence_with_copy_on_write_of_its_last_page():
     fork = parent.copy()
     fork[-1] = fresh
     base.block_tables[1, :n_pages] = fork
-    run = GpuRun(base)
+    run = DeviceRun(base)
     try:
         k_ref, v_ref = base.k_pool.copy(), base.v_pool.copy()
         ap.kv_copy_pages(run.pool, run.pool, [fresh], [int(parent[-1])])
@@ -340,7 +340,7 @@ def test_decode_stream_cut_into_more_than_32_partials():
     one item per SM, so the in-kernel LSE merge takes its chunked path (more partials than a warp has
     lanes).  Every output against the oracle."""
     b = decode_batch(107, (8, 1, 128), [120000], pool_factor=1.05)
-    run = GpuRun(b)
+    run = DeviceRun(b)
     try:
         ex = ap.plan_export(run.plan)
         assert int(ex["merge_entries"][:, 3].max()) > 32, "the plan does not reach the chunked merge"
@@ -358,7 +358,7 @@ def test_decode_more_items_per_cta_than_the_shared_memory_list_holds():
     CTA keeps in shared memory, so the rest come from global memory.  Every output against the oracle."""
     rng = np.random.default_rng(11)
     b = decode_batch(110, W.SHAPE_8B, rng.integers(1, 49, size=1500))
-    run = GpuRun(b)
+    run = DeviceRun(b)
     try:
         ex = ap.plan_export(run.plan)
         assert int(np.diff(ex["cta_begin"]).max()) > 32, "no CTA holds more than 32 items"
@@ -454,7 +454,7 @@ def test_empty_and_skipped_sequences():
 
 def test_workspace_too_small_is_reported():
     b = decode_batch(106, W.SHAPE_8B, [30000])
-    run = GpuRun(b)
+    run = DeviceRun(b)
     assert run.workspace_bytes > 0
     with pytest.raises(ap.ApError) as e:
         ap.attention_iteration(run.pool, run.plan, run.q, run.out, run.lse, run.workspace, run.workspace_bytes - 1)
@@ -490,7 +490,7 @@ def test_host_buffer_iteration_against_the_oracle():
                     np.array([77, 9000, 400, 1300, 16], np.int32), 1.3)
     k_ref, v_ref = oracle_pools(b)
     ref_out, ref_lse = oracle.attention(k_ref, v_ref, b.q_lens, b.ctx_lens, b.block_tables, b.q)
-    run = GpuRun(b)
+    run = DeviceRun(b)
     try:
         assert run.info["merge_entries"] > 0
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).pin_memory()
@@ -505,7 +505,7 @@ def test_host_buffer_iteration_against_the_oracle():
         host_out, host_lse = out.numpy().view(np.uint16).copy(), lse.numpy().copy()
     finally:
         run.close()
-    run = GpuRun(b)
+    run = DeviceRun(b)
     try:
         run.append(); run.attend()
         assert run.status() == 0
@@ -616,7 +616,7 @@ def test_bounded_wait_times_out_and_the_pool_recovers():
     import oracle
     from harness import compare_outputs, oracle_pools
     b = decode_batch(120, W.SHAPE_8B, [20000, 9001, 333])
-    run = GpuRun(b)
+    run = DeviceRun(b)
     try:
         assert run.info["merge_entries"] > 0
         with pytest.raises(ap.ApError):

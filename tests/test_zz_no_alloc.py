@@ -22,7 +22,7 @@ import paper_2604_07144_b200 as ap
 from paper_2604_07144_b200 import binding as B
 from paper_2604_07144_b200 import workloads as W
 
-from harness import GpuRun, LSE_RTOL, OUT_ATOL, oracle_pools, to_bits
+from harness import DeviceRun, LSE_RTOL, OUT_ATOL, oracle_pools, to_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -69,8 +69,8 @@ def _same(got, ref):
 def test_static_workspace_matches_caller_workspace_twice_in_a_row():
     assert ap.static_workspace_bytes() == 8 << 20
     # long contexts: every (row, kv head) stream is cut, so partials and the merge are exercised
-    a = GpuRun(_decode_batch(901, [20000, 9001, 333, 64]))
-    b = GpuRun(_decode_batch(902, [15000, 12000, 17]))
+    a = DeviceRun(_decode_batch(901, [20000, 9001, 333, 64]))
+    b = DeviceRun(_decode_batch(902, [15000, 12000, 17]))
     try:
         assert a.info["merge_entries"] > 0 and b.info["merge_entries"] > 0
         assert 0 < a.workspace_bytes <= ap.static_workspace_bytes()
@@ -106,7 +106,7 @@ def test_static_workspace_with_a_mixed_plan_run_side_by_side():
     # this entry point still allocates nothing.
     batch = W._assemble("static_ws_mixed", W.SHAPE_8B, W.make_rng(904), np.array([140, 1, 1, 1], np.int32),
                         np.array([500, 9000, 4000, 33], np.int32), 1.3)
-    run = GpuRun(batch, side_by_side=3)
+    run = DeviceRun(batch, side_by_side=3)
     try:
         assert run.info["side_by_side"] == 1 and run.info["merge_entries"] > 0
         ref = _reference(run)
@@ -124,7 +124,7 @@ def test_static_workspace_small_plan_and_argument_checks():
     # arguments are refused before anything is launched.  (A plan larger than
     # the 8 MiB array cannot be produced by the planner on 148 SMs, so the
     # size rule is checked on the plan's own number.)
-    run = GpuRun(_decode_batch(903, [40, 700]))
+    run = DeviceRun(_decode_batch(903, [40, 700]))
     try:
         assert run.workspace_bytes <= ap.static_workspace_bytes()
         run.append()
