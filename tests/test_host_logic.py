@@ -218,6 +218,40 @@ def test_side_by_side_planning():
     ap.kv_pool_destroy(pool)
 
 
+def _mixed(shape, n_prefill, n_decode, dec_hi=4096, seed=77):
+    rng = W.make_rng(seed)
+    prefix = rng.g.integers(0, 4097, size=n_prefill)
+    dec = rng.g.integers(256, dec_hi + 1, size=n_decode)
+    q_lens = np.concatenate([np.full(n_prefill, 512), np.ones(n_decode)]).astype(np.int32)
+    ctx = np.concatenate([prefix + 512, dec]).astype(np.int32)
+    return W._assemble("mixed", shape, rng, q_lens, ctx, with_pool=False)
+
+
+def test_side_by_side_decision_at_other_shapes_and_mixes():
+    """The planner's decision for mixes other than config 3, as measured on B200 (the planner's choice beat
+    the sequential dispatch by 7-11 % in each side-by-side case below, and sequential was right for d = 64):
+    70B shape -> a few dozen decode CTAs; a decode-heavy 8B mix -> the cap of 0.7 #SM; a prefill-heavy one ->
+    a handful of CTAs; the d = 64 shape, whose small TMA requests feed an SM too slowly, stays sequential."""
+    def plan_info(batch):
+        pool = ap.kv_pool_create(batch.num_pages, batch.num_kv_heads, batch.head_dim, device=-1)
+        plan = ap.plan_create(pool, batch.q_lens, batch.ctx_lens, batch.block_tables, batch.num_q_heads)
+        info, pred = ap.plan_get_info(plan), ap.plan_predict(plan)
+        ap.plan_destroy(plan)
+        ap.kv_pool_destroy(pool)
+        return info, pred
+    i, p = plan_info(_mixed(W.SHAPE_70B, 8, 120))
+    assert i["side_by_side"] == 1 and 30 <= i["decode_ctas"] <= 60 and i["decode_head_block"] == 4
+    assert 380 <= p["model_step_us"] <= 520                     # measured 457 us
+    i, p = plan_info(_mixed(W.SHAPE_8B, 2, 300))
+    assert i["side_by_side"] == 1 and i["decode_ctas"] == 103
+    assert 340 <= p["model_step_us"] <= 520                     # measured 402 us
+    i, p = plan_info(_mixed(W.SHAPE_8B, 14, 40))
+    assert i["side_by_side"] == 1 and 12 <= i["decode_ctas"] <= 30
+    assert 290 <= p["model_step_us"] <= 400                     # measured 342 us
+    i, _ = plan_info(_mixed(W.SHAPE_S1, 8, 400, dec_hi=8192))
+    assert i["side_by_side"] == 0 and i["decode_head_block"] == 2
+
+
 def test_copy_pages_validation_on_host_pools():
     """ap_kv_copy_pages checks its lists on the host before anything is queued."""
     a, b = host_pool(20), host_pool(30)
