@@ -47,10 +47,10 @@ UNIT = "KV-tokens/s"
 # workload (ncu captures summarised under profiles/), keyed by (kernel, config, hash of
 # the kernel's source file the counters were taken from); a changed kernel reports null.
 NCU_TRAFFIC = {
-    # profiles/decode_splitk_config2.md: 536.9 MB read + 5.2 MB written per launch (algorithmic 535.0 MB)
-    ("decode_splitk", 2, "ca0a806fd24723da"): 542.1e6,
-    # profiles/prefill_tcgen05_config3.md: 149.6 MB read + 18.8 MB written per launch (K/V re-reads are served by the L2)
-    ("prefill_tcgen05", 3, "d85139c575f9e37a"): 168.4e6,
+    # profiles/decode_splitk_config2.md: 536.5 MB read + 3.8 MB written per launch (algorithmic 535.0 MB)
+    ("decode_splitk", 2, "e7670ad945da38e5"): 540.3e6,
+    # profiles/prefill_tcgen05_config3.md: 149.4 MB read + 18.0 MB written per launch (K/V re-reads are served by the L2)
+    ("prefill_tcgen05", 3, "080aa46481f9814f"): 167.4e6,
 }
 
 

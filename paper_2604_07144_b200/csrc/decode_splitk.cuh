@@ -313,6 +313,9 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
         int32_t cur = lane < item.page_count ? __ldg(bt_flat + item.bt_offset + item.page_begin + lane) : 0;
         griddep_wait();      // after the first block-table entries are on their way
         const uint32_t page_bytes = (uint32_t)(2 * HB * Cfg::kTileBytes);   // K and V tiles of one page of the block
+        // a decode stream is read once: its lines should be the first to leave the L2 (next to a prefill
+        // kernel, whose units read the same K/V tiles again and again, they would otherwise push those out)
+        const uint64_t stream_once = l2_policy_evict_first();
         for (int n = 0; item.page_count > 0; ++n) {
             const int32_t *bt = bt_flat + item.bt_offset + item.page_begin;
             const int npages = item.page_count;
@@ -356,8 +359,8 @@ __device__ __forceinline__ void decode_cta(const CUtensorMap &k_map, const CUten
                         }
                         // one request per plane: the HB tiles of this page that belong to the item's kv heads
                         const int group = (page * Hkv + item.kv_head) * 2;
-                        tma_load_4d(st + lane * HB * Cfg::kTileBytes, &k_map, &full[stage], 0, 0, 0, group);
-                        tma_load_4d(st + (kTPS + lane * HB) * Cfg::kTileBytes, &v_map, &full[stage], 0, 0, 0, group);
+                        tma_load_4d_hint(st + lane * HB * Cfg::kTileBytes, &k_map, &full[stage], 0, 0, 0, group, stream_once);
+                        tma_load_4d_hint(st + (kTPS + lane * HB) * Cfg::kTileBytes, &v_map, &full[stage], 0, 0, 0, group, stream_once);
                     }
                     advance();
                 }
